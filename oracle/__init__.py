@@ -1,0 +1,132 @@
+"""ctypes front end of the DES-LOC CPU oracle (``desloc_oracle.c``).
+
+TEST INFRASTRUCTURE, NOT THE PRODUCT: only the test-suite, the smoke check and
+the benchmark's CPU-baseline leg import this package.  It builds the C file
+with gcc on first use and forwards numpy arrays to it; all of the method's
+arithmetic lives in the C file (Algorithms 1-3 of the paper, plus the
+post-average ordering of Algorithms 4-5).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+ADAM, ADOPT, SGDM = 0, 1, 2
+SYNC_X, SYNC_U, SYNC_V = 1, 2, 4
+FLAG_ADOPT_NORM_CLIP = 1
+FLAG_POST_AVERAGE = 2
+FLAG_ADOPT_AVG_NORMALISER = 4
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "desloc_oracle.c")
+_LIB = os.path.join(_HERE, "libdesloc_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+class OracleCfg(ctypes.Structure):
+    _fields_ = [
+        ("M", ctypes.c_int32),
+        ("opt", ctypes.c_int32),
+        ("beta1", ctypes.c_double),
+        ("beta2", ctypes.c_double),
+        ("eps", ctypes.c_double),
+        ("weight_decay", ctypes.c_double),
+        ("clip_rho", ctypes.c_double),
+        ("Kx", ctypes.c_int32),
+        ("Ku", ctypes.c_int32),
+        ("Kv", ctypes.c_int32),
+        ("flags", ctypes.c_uint32),
+    ]
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O2, no fast-math) if it is stale."""
+    with _lock:
+        stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+        if force or stale:
+            tmp = _LIB + f".tmp{os.getpid()}"
+            subprocess.check_call(
+                ["gcc", "-O2", "-std=c99", "-ffp-contract=off", "-Wall", "-Wextra", "-shared",
+                 "-fPIC", "-o", tmp, _SRC, "-lm"])
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        L.desloc_oracle_sync_mask.restype = ctypes.c_uint32
+        L.desloc_oracle_sync_mask.argtypes = [ctypes.c_int32] * 4 + [ctypes.c_int64]
+        L.desloc_oracle_step.restype = ctypes.c_uint32
+        L.desloc_oracle_step.argtypes = [
+            ctypes.POINTER(OracleCfg), ctypes.c_int64, ctypes.c_double, ctypes.c_double,
+            ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+            ctypes.c_void_p]
+        L.desloc_oracle_run.restype = None
+        L.desloc_oracle_run.argtypes = [
+            ctypes.POINTER(OracleCfg), ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p,
+            ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p,
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        _lib = L
+    return _lib
+
+
+def make_cfg(M, opt, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0, clip_rho=0.0,
+             Kx=1, Ku=1, Kv=1, flags=0) -> OracleCfg:
+    return OracleCfg(int(M), int(opt), float(beta1), float(beta2), float(eps),
+                     float(weight_decay), float(clip_rho), int(Kx), int(Ku), int(Kv), int(flags))
+
+
+def sync_mask(opt, Kx, Ku, Kv, t) -> int:
+    return int(lib().desloc_oracle_sync_mask(int(opt), int(Kx), int(Ku), int(Kv), int(t)))
+
+
+def _check(a, M, name, allow_none=False):
+    if a is None:
+        if allow_none:
+            return None
+        raise ValueError(f"{name} is required")
+    if not (isinstance(a, np.ndarray) and a.dtype == np.float32 and a.ndim == 2
+            and a.shape[0] == M and a.flags["C_CONTIGUOUS"]):
+        raise ValueError(f"{name} must be a C-contiguous float32 array of shape [M, n]")
+    return a.ctypes.data
+
+
+def step(cfg: OracleCfg, t: int, lr: float, x, u, v, g, clip_bound: float = 0.0) -> int:
+    """One step in place on float32 arrays of shape [M, n]; returns the sync mask."""
+    M = cfg.M
+    px, pu, pg = _check(x, M, "x"), _check(u, M, "u"), _check(g, M, "g")
+    pv = _check(v, M, "v", allow_none=(cfg.opt == SGDM))
+    n = x.shape[1]
+    if u.shape != x.shape or g.shape != x.shape or (v is not None and v.shape != x.shape):
+        raise ValueError("x, u, v, g must share one shape")
+    return int(lib().desloc_oracle_step(ctypes.byref(cfg), int(t), float(lr), float(clip_bound),
+                                        n, n, px, pu, pv, pg))
+
+
+def run(cfg: OracleCfg, t0: int, lrs, x, u, v, g, clip_bounds=None):
+    """T = len(lrs) steps in place; g has shape [T, M, n].  Returns the mask of every step."""
+    M = cfg.M
+    lrs = np.ascontiguousarray(lrs, dtype=np.float64)
+    T = lrs.shape[0]
+    if not (g.dtype == np.float32 and g.ndim == 3 and g.shape[0] == T and g.shape[1] == M
+            and g.flags["C_CONTIGUOUS"] and g.shape[2] == x.shape[1]):
+        raise ValueError("g must be a C-contiguous float32 array of shape [T, M, n]")
+    px, pu = _check(x, M, "x"), _check(u, M, "u")
+    pv = _check(v, M, "v", allow_none=(cfg.opt == SGDM))
+    cb = None
+    if clip_bounds is not None:
+        cb = np.ascontiguousarray(clip_bounds, dtype=np.float64)
+        assert cb.shape[0] == T
+    masks = np.zeros(T, dtype=np.uint32)
+    n = x.shape[1]
+    lib().desloc_oracle_run(ctypes.byref(cfg), int(t0), T, lrs.ctypes.data,
+                            cb.ctypes.data if cb is not None else None, n, n, px, pu, pv,
+                            g.ctypes.data, masks.ctypes.data)
+    return masks
