@@ -1,0 +1,180 @@
+/*
+ * desloc.h -- C ABI of the DES-LOC optimizer-step library for NVIDIA B200 (sm_100a).
+ *
+ * DES-LOC (Desynced Low Communication Adaptive Optimizers): M workers each take
+ * local Adam, ADOPT or SGD-momentum steps; the parameters x and the optimizer
+ * states u (first moment / momentum) and v (second moment) are averaged across
+ * workers on independent periods K_x, K_u, K_v (Algorithm 1 of the paper).
+ *
+ * This library keeps all M worker replicas in ONE GPU's memory.  One call to
+ * desloc_step() runs one step t of Algorithm 1 for all workers: a single
+ * memory-bound kernel reads g, x, u, v of every replica once, clips the
+ * gradient, averages the arrays whose period divides t in registers (fixed
+ * order m = 0..M-1), applies the per-worker update and writes x, u, v back.
+ * A sync step therefore moves the same bytes as a local step; there is no
+ * separate averaging pass and no collective.
+ *
+ * Conventions
+ *   - Every pointer named "device" must be valid on the CUDA device given to
+ *     desloc_create(); every other pointer is host memory.
+ *   - x, u, v are fp32 and caller-owned; the library updates them in place and
+ *     borrows the pointers for the lifetime of the context.  Gradients are
+ *     fp32 or bf16, read-only, and may live somewhere else at every step.
+ *   - All functions return DESLOC_OK (0) or a negative desloc_status; nothing
+ *     throws, aborts or prints.  desloc_last_cuda_error() gives the CUDA error
+ *     behind a DESLOC_E_CUDA.  There is no CPU fallback: without a usable
+ *     device every compute entry point returns DESLOC_E_CUDA.
+ *   - One context may be used by one host thread at a time.
+ */
+#ifndef DESLOC_H_
+#define DESLOC_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define DESLOC_API __attribute__((visibility("default")))
+#else
+#define DESLOC_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DESLOC_MAX_M 64 /* largest worker count a context accepts */
+
+typedef struct desloc_ctx desloc_ctx; /* opaque, library-owned */
+
+typedef enum {
+    DESLOC_ADAM = 0,  /* Algorithm 2 */
+    DESLOC_ADOPT = 1, /* Algorithm 3 */
+    DESLOC_SGDM = 2   /* Algorithm 1 with N = 1 state: u = beta u + (1-beta) g, x = x - eta u */
+} desloc_opt_t;
+
+typedef enum { DESLOC_F32 = 0, DESLOC_BF16 = 1 } desloc_dtype_t;
+
+/* Bits of the sync mask: which arrays are averaged over the workers at a step. */
+enum { DESLOC_SYNC_X = 1, DESLOC_SYNC_U = 2, DESLOC_SYNC_V = 4 };
+
+enum {
+    /* ADOPT only: clamp the normalised gradient g / max(sqrt(v), eps) to +-clip_bound_t,
+       the per-step bound handed to desloc_step().  Not part of Algorithm 3; the ADOPT
+       optimizer the paper builds on has it, and with v_{-1} = 0 it keeps step 0 finite. */
+    DESLOC_FLAG_ADOPT_NORM_CLIP = 1u,
+    /* Average AFTER the local update instead of before it (the ordering of Algorithms 4
+       and 5): on a sync step the new u / v / x are averaged and every worker stores the mean. */
+    DESLOC_FLAG_POST_AVERAGE = 2u
+};
+
+typedef enum {
+    DESLOC_OK = 0,
+    DESLOC_E_NULL = -1,    /* a required pointer is NULL */
+    DESLOC_E_RANGE = -2,   /* M, a period, a beta, eps, weight decay, numel or t out of range */
+    DESLOC_E_INVALID = -3, /* unknown optimizer / dtype / flag, or a flag the optimizer lacks */
+    DESLOC_E_NOMEM = -4,   /* host or device allocation failed */
+    DESLOC_E_CUDA = -5     /* a CUDA call failed; see desloc_last_cuda_error() */
+} desloc_status;
+
+/* The "Require" block of Algorithms 1-3: everything fixed for a run.  Plain data, copied
+   by desloc_create(). */
+typedef struct {
+    int32_t M;              /* workers, 1..DESLOC_MAX_M */
+    int32_t num_tensors;    /* >= 1: the model is a list of tensors */
+    const int64_t *numel;   /* host, [num_tensors], each >= 1 */
+    int32_t opt;            /* desloc_opt_t */
+    int32_t grad_dtype;     /* desloc_dtype_t of the gradients */
+    float beta1, beta2;     /* decay factors in [0, 1); SGDM uses beta1 only */
+    float eps;              /* Adam: lambda, enters as sqrt(v + lambda^2); ADOPT: epsilon in
+                               max(sqrt(v), epsilon); >= 0 */
+    float weight_decay;     /* >= 0, decoupled: x* (1 - eta_t wd) - d_t.  The paper uses 0. */
+    float clip_rho;         /* coordinate clip radius rho of Section 3.1; <= 0 switches it off */
+    int32_t Kx, Ku, Kv;     /* sync periods, >= 0; 0 = never (K = infinity); SGDM ignores Kv */
+    uint32_t flags;         /* DESLOC_FLAG_* */
+} desloc_config;
+
+/*
+ * Which arrays Algorithm 1 averages at step t (t counts from 0, so t = 0 syncs every array
+ * with a non-zero period): bit X iff Kx > 0 and t mod Kx == 0, likewise U and V; the V bit is
+ * always clear for SGDM.  Pure host function; cfg->numel is not read.  Returns 0 for a NULL
+ * cfg or t < 0.
+ */
+DESLOC_API uint32_t desloc_sync_mask(const desloc_config *cfg, int64_t t);
+
+/*
+ * Create a context for `cfg` on CUDA device `cuda_device`.
+ *   x, u, v : host arrays of M*num_tensors DEVICE pointers, entry [m*num_tensors + k] is worker
+ *             m's copy of tensor k (numel[k] fp32 values).  v may be NULL for SGDM.  No two
+ *             entries may overlap.  The pointer arrays themselves are copied; the tensors are
+ *             borrowed until desloc_destroy().  Any alignment is accepted: tensors whose
+ *             pointers are all 16-byte aligned take the vector path, the rest a scalar path.
+ * Validates everything before touching the device.  Allocates the context, its device-side
+ * pointer and chunk tables, and a few pinned staging buffers -- nothing is allocated later.
+ * Initial state is whatever the buffers hold (Algorithm 1 starts every worker from the same
+ * x_0 and zero states).
+ */
+DESLOC_API int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *const *x, float *const *u,
+                  float *const *v, int cuda_device);
+
+/*
+ * One step t of Algorithm 1 (Algorithm 2 / 3 / SGDM per cfg.opt) for all M workers.
+ *   t            : step counter, >= 0; decides the sync mask via desloc_sync_mask().
+ *   lr_t         : eta_t, the learning rate of this step (the schedule is the caller's).
+ *   clip_bound_t : bound for DESLOC_FLAG_ADOPT_NORM_CLIP at this step; ignored otherwise.
+ *   grads        : host array of M*num_tensors DEVICE pointers (same indexing as x) to
+ *                  gradients of cfg.grad_dtype; read-only; may differ from call to call.
+ *   stream       : a cudaStream_t (NULL = default stream).  The call only enqueues work and
+ *                  never synchronises the device.
+ *   mask_out     : if not NULL receives the sync mask that was applied.
+ * Errors: a failed launch is returned by this call; an asynchronous execution error surfaces
+ * in a later call or at the caller's next synchronisation.
+ */
+DESLOC_API int desloc_step(desloc_ctx *ctx, int64_t t, float lr_t, float clip_bound_t,
+                const void *const *grads, void *stream, uint32_t *mask_out);
+
+/* As desloc_step() but with the sync mask given by the caller instead of derived from t
+   (used to time or test one sync pattern in isolation).  mask bits outside X|U|V, or V for
+   SGDM, are rejected with DESLOC_E_INVALID.  Counters are updated as for desloc_step(). */
+DESLOC_API int desloc_step_masked(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
+                       const void *const *grads, void *stream);
+
+/* Release the context and everything it allocated.  The caller's tensors are untouched.
+   NULL is a no-op returning DESLOC_OK. */
+DESLOC_API int desloc_destroy(desloc_ctx *ctx);
+
+/* out[0..3] = steps taken, x-syncs, u-syncs, v-syncs (the per-array communication counts a
+   distributed run of the same schedule would pay; Section 5.1 "Metrics"). */
+DESLOC_API int desloc_get_counters(const desloc_ctx *ctx, int64_t out[4]);
+
+/* Kernels launched by this context so far (one per step on the main path). */
+DESLOC_API int64_t desloc_get_launch_count(const desloc_ctx *ctx);
+
+/*
+ * Grid shape of the step kernel: ctas_per_sm = 0 (default) launches one thread block per work
+ * item (a chunk, or a (worker, chunk) pair on local steps); 1..32 launches a persistent grid
+ * of that many blocks per SM which stride over the items.  Results do not depend on it.
+ */
+DESLOC_API int desloc_set_launch_shape(desloc_ctx *ctx, int32_t ctas_per_sm);
+
+/*
+ * Multi-tensor plan: how the tensor list is cut into the fixed-size chunks that thread
+ * blocks work through.  Host-only.  Writes up to `cap` chunks as triples
+ * (tensor index, first element, element count) into `out` (3*cap int64) and returns the total
+ * number of chunks the list needs (which may exceed cap), or a negative desloc_status.
+ * Every tensor starts a new chunk; chunks of a tensor are `chunk_elems` long except the last.
+ */
+DESLOC_API int64_t desloc_plan_chunks(const int64_t *numel, int32_t num_tensors, int64_t chunk_elems,
+                           int64_t *out, int64_t cap);
+
+/* Elements per chunk used by contexts of this build. */
+DESLOC_API int64_t desloc_chunk_elems(void);
+
+/* Static description of a status code; never NULL. */
+DESLOC_API const char *desloc_strerror(int status);
+
+/* The last CUDA error code (cudaError_t as int) seen by this context, 0 if none. */
+DESLOC_API int desloc_last_cuda_error(const desloc_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DESLOC_H_ */

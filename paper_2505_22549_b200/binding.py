@@ -1,0 +1,208 @@
+"""ctypes binding of libdesloc.so: the functions of include/desloc.h under the same names.
+
+Argument marshalling only -- every step of the DES-LOC update runs in the CUDA kernels of
+the library.  There is no fallback: if the library cannot be loaded, importing this module
+raises.  Device pointers are plain integers (e.g. ``tensor.data_ptr()``); streams are the
+integer ``cudaStream_t`` (e.g. ``torch.cuda.current_stream().cuda_stream``).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "lib", "libdesloc.so")
+
+DESLOC_ADAM, DESLOC_ADOPT, DESLOC_SGDM = 0, 1, 2
+DESLOC_F32, DESLOC_BF16 = 0, 1
+DESLOC_SYNC_X, DESLOC_SYNC_U, DESLOC_SYNC_V = 1, 2, 4
+DESLOC_FLAG_ADOPT_NORM_CLIP, DESLOC_FLAG_POST_AVERAGE = 1, 2
+DESLOC_OK, DESLOC_E_NULL, DESLOC_E_RANGE, DESLOC_E_INVALID, DESLOC_E_NOMEM, DESLOC_E_CUDA = \
+    0, -1, -2, -3, -4, -5
+DESLOC_MAX_M = 64
+
+OPT_BY_NAME = {"adam": DESLOC_ADAM, "adopt": DESLOC_ADOPT, "sgdm": DESLOC_SGDM}
+DTYPE_BY_NAME = {"f32": DESLOC_F32, "bf16": DESLOC_BF16}
+
+
+class DeslocConfig(ctypes.Structure):
+    """Mirror of ``desloc_config``."""
+    _fields_ = [
+        ("M", ctypes.c_int32),
+        ("num_tensors", ctypes.c_int32),
+        ("numel", ctypes.POINTER(ctypes.c_int64)),
+        ("opt", ctypes.c_int32),
+        ("grad_dtype", ctypes.c_int32),
+        ("beta1", ctypes.c_float),
+        ("beta2", ctypes.c_float),
+        ("eps", ctypes.c_float),
+        ("weight_decay", ctypes.c_float),
+        ("clip_rho", ctypes.c_float),
+        ("Kx", ctypes.c_int32),
+        ("Ku", ctypes.c_int32),
+        ("Kv", ctypes.c_int32),
+        ("flags", ctypes.c_uint32),
+    ]
+
+
+class DeslocError(RuntimeError):
+    def __init__(self, status: int, where: str, cuda_error: int = 0):
+        self.status = status
+        self.cuda_error = cuda_error
+        msg = f"{where}: {desloc_strerror(status)} (status {status}"
+        msg += f", cudaError {cuda_error})" if cuda_error else ")"
+        super().__init__(msg)
+
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2505_22549_b200.build` "
+        "(there is no CPU or PyTorch fallback for the DES-LOC step)")
+_lib = ctypes.CDLL(LIB_PATH)
+
+_P = ctypes.c_void_p
+_PP = ctypes.POINTER(ctypes.c_void_p)
+_lib.desloc_sync_mask.restype = ctypes.c_uint32
+_lib.desloc_sync_mask.argtypes = [ctypes.POINTER(DeslocConfig), ctypes.c_int64]
+_lib.desloc_create.restype = ctypes.c_int
+_lib.desloc_create.argtypes = [ctypes.POINTER(_P), ctypes.POINTER(DeslocConfig), _PP, _PP, _PP,
+                               ctypes.c_int]
+_lib.desloc_step.restype = ctypes.c_int
+_lib.desloc_step.argtypes = [_P, ctypes.c_int64, ctypes.c_float, ctypes.c_float, _PP, _P,
+                             ctypes.POINTER(ctypes.c_uint32)]
+_lib.desloc_step_masked.restype = ctypes.c_int
+_lib.desloc_step_masked.argtypes = [_P, ctypes.c_uint32, ctypes.c_float, ctypes.c_float, _PP, _P]
+_lib.desloc_destroy.restype = ctypes.c_int
+_lib.desloc_destroy.argtypes = [_P]
+_lib.desloc_get_counters.restype = ctypes.c_int
+_lib.desloc_get_counters.argtypes = [_P, ctypes.POINTER(ctypes.c_int64)]
+_lib.desloc_get_launch_count.restype = ctypes.c_int64
+_lib.desloc_get_launch_count.argtypes = [_P]
+_lib.desloc_set_launch_shape.restype = ctypes.c_int
+_lib.desloc_set_launch_shape.argtypes = [_P, ctypes.c_int32]
+_lib.desloc_plan_chunks.restype = ctypes.c_int64
+_lib.desloc_plan_chunks.argtypes = [ctypes.POINTER(ctypes.c_int64), ctypes.c_int32,
+                                    ctypes.c_int64, ctypes.POINTER(ctypes.c_int64),
+                                    ctypes.c_int64]
+_lib.desloc_chunk_elems.restype = ctypes.c_int64
+_lib.desloc_chunk_elems.argtypes = []
+_lib.desloc_strerror.restype = ctypes.c_char_p
+_lib.desloc_strerror.argtypes = [ctypes.c_int]
+_lib.desloc_last_cuda_error.restype = ctypes.c_int
+_lib.desloc_last_cuda_error.argtypes = [_P]
+
+
+def raw_lib() -> ctypes.CDLL:
+    """The loaded shared library (for tests that check the exported symbols)."""
+    return _lib
+
+
+def make_config(M: int, numel: Sequence[int], opt, grad_dtype, beta1=0.9, beta2=0.999, eps=1e-8,
+                weight_decay=0.0, clip_rho=0.0, Kx=1, Ku=1, Kv=1, flags=0) -> DeslocConfig:
+    """Fill a ``desloc_config``.  The numel array is kept alive on the returned object."""
+    opt = OPT_BY_NAME.get(opt, opt)
+    grad_dtype = DTYPE_BY_NAME.get(grad_dtype, grad_dtype)
+    arr = (ctypes.c_int64 * len(numel))(*[int(n) for n in numel])
+    cfg = DeslocConfig(int(M), len(numel), ctypes.cast(arr, ctypes.POINTER(ctypes.c_int64)),
+                       int(opt), int(grad_dtype), float(beta1), float(beta2), float(eps),
+                       float(weight_decay), float(clip_rho), int(Kx), int(Ku), int(Kv), int(flags))
+    cfg._numel_keepalive = arr
+    return cfg
+
+
+def _ptr_array(ptrs: Optional[Sequence[int]]):
+    if ptrs is None:
+        return None
+    return (ctypes.c_void_p * len(ptrs))(*[int(p) if p else None for p in ptrs])
+
+
+def desloc_strerror(status: int) -> str:
+    return _lib.desloc_strerror(int(status)).decode()
+
+
+def desloc_sync_mask(cfg: DeslocConfig, t: int) -> int:
+    return int(_lib.desloc_sync_mask(ctypes.byref(cfg) if cfg is not None else None, int(t)))
+
+
+def desloc_create(cfg: DeslocConfig, x: Sequence[int], u: Sequence[int],
+                  v: Optional[Sequence[int]], cuda_device: int) -> int:
+    """Returns the context handle (an integer); raises DeslocError on failure."""
+    handle = ctypes.c_void_p()
+    rc = _lib.desloc_create(ctypes.byref(handle), ctypes.byref(cfg) if cfg is not None else None,
+                            _ptr_array(x), _ptr_array(u), _ptr_array(v), int(cuda_device))
+    if rc != DESLOC_OK:
+        raise DeslocError(rc, "desloc_create")
+    return handle.value
+
+
+def desloc_step(ctx: int, t: int, lr_t: float, clip_bound_t: float, grads, stream: int = 0) -> int:
+    """One step; returns the sync mask applied.  `grads` is a sequence of device pointers or a
+    ready ctypes pointer array (see ptr_array) to skip re-marshalling in a hot loop."""
+    g = grads if isinstance(grads, ctypes.Array) else _ptr_array(grads)
+    mask = ctypes.c_uint32(0)
+    rc = _lib.desloc_step(ctx, int(t), float(lr_t), float(clip_bound_t), g, stream or None,
+                          ctypes.byref(mask))
+    if rc != DESLOC_OK:
+        raise DeslocError(rc, "desloc_step", _lib.desloc_last_cuda_error(ctx))
+    return int(mask.value)
+
+
+def desloc_step_masked(ctx: int, mask: int, lr_t: float, clip_bound_t: float, grads,
+                       stream: int = 0) -> None:
+    g = grads if isinstance(grads, ctypes.Array) else _ptr_array(grads)
+    rc = _lib.desloc_step_masked(ctx, int(mask), float(lr_t), float(clip_bound_t), g,
+                                 stream or None)
+    if rc != DESLOC_OK:
+        raise DeslocError(rc, "desloc_step_masked", _lib.desloc_last_cuda_error(ctx))
+
+
+def desloc_destroy(ctx: Optional[int]) -> None:
+    rc = _lib.desloc_destroy(ctx)
+    if rc != DESLOC_OK:
+        raise DeslocError(rc, "desloc_destroy")
+
+
+def desloc_get_counters(ctx: int):
+    out = (ctypes.c_int64 * 4)()
+    rc = _lib.desloc_get_counters(ctx, out)
+    if rc != DESLOC_OK:
+        raise DeslocError(rc, "desloc_get_counters")
+    return [int(a) for a in out]
+
+
+def desloc_get_launch_count(ctx: int) -> int:
+    return int(_lib.desloc_get_launch_count(ctx))
+
+
+def desloc_set_launch_shape(ctx: int, ctas_per_sm: int) -> None:
+    rc = _lib.desloc_set_launch_shape(ctx, int(ctas_per_sm))
+    if rc != DESLOC_OK:
+        raise DeslocError(rc, "desloc_set_launch_shape")
+
+
+def desloc_chunk_elems() -> int:
+    return int(_lib.desloc_chunk_elems())
+
+
+def desloc_plan_chunks(numel: Sequence[int], chunk_elems: int, cap: Optional[int] = None):
+    """Returns (total_chunks, [(tensor, start, count), ...] up to cap)."""
+    arr = (ctypes.c_int64 * max(1, len(numel)))(*[int(n) for n in numel])
+    total = _lib.desloc_plan_chunks(arr, len(numel), int(chunk_elems), None, 0)
+    if total < 0:
+        raise DeslocError(int(total), "desloc_plan_chunks")
+    cap = total if cap is None else min(cap, total)
+    out = (ctypes.c_int64 * max(1, 3 * cap))()
+    total2 = _lib.desloc_plan_chunks(arr, len(numel), int(chunk_elems), out, cap)
+    assert total2 == total
+    return int(total), [(int(out[3 * i]), int(out[3 * i + 1]), int(out[3 * i + 2]))
+                        for i in range(cap)]
+
+
+def ptr_array(ptrs: Sequence[int]):
+    """A reusable ctypes array of device pointers for desloc_step()."""
+    return _ptr_array(ptrs)
+
+
+def desloc_last_cuda_error(ctx: int) -> int:
+    return int(_lib.desloc_last_cuda_error(ctx))

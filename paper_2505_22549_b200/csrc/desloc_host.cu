@@ -1,0 +1,402 @@
+// Host side of the DES-LOC library: the C ABI of include/desloc.h, argument validation, the
+// sync schedule (Algorithm 1's "t mod K = 0" tests), the multi-tensor chunk plan and the
+// launcher that picks one kernel instantiation per step.  No torch types, no CPU compute path.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdint>
+#include <cstdlib>
+#include <cstring>
+#include <limits>
+#include <new>
+#include <vector>
+
+#include "../../include/desloc.h"
+#include "desloc_inst.cuh"
+
+namespace desloc {
+
+const void *lookup_step_kernel(int opt, bool post, bool bf16, int mt, int mask) {
+    if (mask == 0) {
+        // Local step: the same code for either ordering and any M.
+        if (opt == OPT_ADAM) return lookup_adam_pre(bf16, 1, 0);
+        if (opt == OPT_ADOPT) return lookup_adopt_pre(bf16, 1, 0);
+        if (opt == OPT_SGDM) return lookup_sgdm_pre(bf16, 1, 0);
+        return nullptr;
+    }
+    if (opt == OPT_ADAM) return post ? lookup_adam_post(bf16, mt, mask) : lookup_adam_pre(bf16, mt, mask);
+    if (opt == OPT_ADOPT) return post ? lookup_adopt_post(bf16, mt, mask) : lookup_adopt_pre(bf16, mt, mask);
+    if (opt == OPT_SGDM) return post ? lookup_sgdm_post(bf16, mt, mask) : lookup_sgdm_pre(bf16, mt, mask);
+    return nullptr;
+}
+
+}  // namespace desloc
+
+namespace {
+
+constexpr int kSlots = 8;  // staging slots for per-step gradient pointer tables
+
+struct Slot {
+    void **host = nullptr;  // pinned
+    void **dev = nullptr;
+    cudaEvent_t done = nullptr;
+    bool in_flight = false;
+};
+
+}  // namespace
+
+struct desloc_ctx {
+    desloc_config cfg{};
+    std::vector<int64_t> numel;
+    int device = 0;
+    int num_sms = 0;
+    int64_t total_elems = 0;
+    int64_t nptr = 0;  // M * num_tensors
+    desloc::Chunk *d_chunks = nullptr;
+    int64_t nchunks = 0;
+    void **d_tables = nullptr;  // [3][nptr] x, u, v
+    Slot slots[kSlots];
+    int next_slot = 0;
+    int cur_slot = -1;           // slot holding the table equal to last_grads
+    std::vector<const void *> last_grads;
+    cudaStream_t last_stream = nullptr;
+    int64_t counters[4] = {0, 0, 0, 0};
+    int64_t launches = 0;
+    int last_cuda_error = 0;
+    int ctas_per_sm = 0;  // 0: one block per work item; > 0: persistent grid of that many per SM
+};
+
+namespace {
+
+int cuda_fail(desloc_ctx *ctx, cudaError_t e) {
+    if (ctx) ctx->last_cuda_error = static_cast<int>(e);
+    (void)cudaGetLastError();  // clear the sticky per-thread error where it can be cleared
+    return DESLOC_E_CUDA;
+}
+
+bool finite_in(float v, float lo, bool lo_incl, float hi, bool hi_incl) {
+    if (!std::isfinite(v)) return false;
+    if (lo_incl ? v < lo : v <= lo) return false;
+    if (hi_incl ? v > hi : v >= hi) return false;
+    return true;
+}
+
+int validate_config(const desloc_config *c) {
+    if (!c) return DESLOC_E_NULL;
+    if (c->opt != DESLOC_ADAM && c->opt != DESLOC_ADOPT && c->opt != DESLOC_SGDM) return DESLOC_E_INVALID;
+    if (c->grad_dtype != DESLOC_F32 && c->grad_dtype != DESLOC_BF16) return DESLOC_E_INVALID;
+    if (c->flags & ~(DESLOC_FLAG_ADOPT_NORM_CLIP | DESLOC_FLAG_POST_AVERAGE)) return DESLOC_E_INVALID;
+    if ((c->flags & DESLOC_FLAG_ADOPT_NORM_CLIP) && c->opt != DESLOC_ADOPT) return DESLOC_E_INVALID;
+    if (c->M < 1 || c->M > DESLOC_MAX_M) return DESLOC_E_RANGE;
+    if (c->num_tensors < 1) return DESLOC_E_RANGE;
+    if (c->Kx < 0 || c->Ku < 0 || c->Kv < 0) return DESLOC_E_RANGE;
+    if (!finite_in(c->beta1, 0.f, true, 1.f, false)) return DESLOC_E_RANGE;
+    if (c->opt != DESLOC_SGDM && !finite_in(c->beta2, 0.f, true, 1.f, false)) return DESLOC_E_RANGE;
+    if (!finite_in(c->eps, 0.f, true, std::numeric_limits<float>::max(), true)) return DESLOC_E_RANGE;
+    if (!finite_in(c->weight_decay, 0.f, true, std::numeric_limits<float>::max(), true)) return DESLOC_E_RANGE;
+    if (std::isnan(c->clip_rho)) return DESLOC_E_RANGE;
+    return DESLOC_OK;
+}
+
+uint32_t mask_at(const desloc_config *c, int64_t t) {
+    uint32_t m = 0;
+    if (c->Kx > 0 && t % c->Kx == 0) m |= DESLOC_SYNC_X;
+    if (c->Ku > 0 && t % c->Ku == 0) m |= DESLOC_SYNC_U;
+    if (c->opt != DESLOC_SGDM && c->Kv > 0 && t % c->Kv == 0) m |= DESLOC_SYNC_V;
+    return m;
+}
+
+void free_ctx(desloc_ctx *ctx) {
+    if (!ctx) return;
+    for (Slot &s : ctx->slots) {
+        if (s.done) cudaEventDestroy(s.done);
+        if (s.host) cudaFreeHost(s.host);
+        if (s.dev) cudaFree(s.dev);
+    }
+    if (ctx->d_chunks) cudaFree(ctx->d_chunks);
+    if (ctx->d_tables) cudaFree(ctx->d_tables);
+    delete ctx;
+}
+
+// Stage the gradient pointer table for this step on `stream`; returns the device table.
+int stage_grads(desloc_ctx *ctx, const void *const *grads, cudaStream_t stream, void ***dev_out) {
+    const size_t bytes = static_cast<size_t>(ctx->nptr) * sizeof(void *);
+    if (ctx->cur_slot >= 0 && stream == ctx->last_stream &&
+        std::memcmp(ctx->last_grads.data(), grads, bytes) == 0) {
+        *dev_out = ctx->slots[ctx->cur_slot].dev;  // same pointers as last step: table is resident
+        return DESLOC_OK;
+    }
+    Slot &s = ctx->slots[ctx->next_slot];
+    if (s.in_flight) {
+        // Re-use of a slot whose kernel was enqueued kSlots table changes ago: wait for it.
+        cudaError_t e = cudaEventSynchronize(s.done);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        s.in_flight = false;
+    }
+    std::memcpy(s.host, grads, bytes);
+    cudaError_t e = cudaMemcpyAsync(s.dev, s.host, bytes, cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    std::memcpy(ctx->last_grads.data(), grads, bytes);
+    ctx->cur_slot = ctx->next_slot;
+    ctx->next_slot = (ctx->next_slot + 1) % kSlots;
+    ctx->last_stream = stream;
+    *dev_out = s.dev;
+    return DESLOC_OK;
+}
+
+int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
+             const void *const *grads, cudaStream_t stream) {
+    const desloc_config &c = ctx->cfg;
+    if (!std::isfinite(lr_t)) return DESLOC_E_RANGE;
+    const bool nclip = (c.flags & DESLOC_FLAG_ADOPT_NORM_CLIP) != 0;
+    if (nclip && !(clip_bound_t >= 0.f)) return DESLOC_E_RANGE;
+    for (int64_t i = 0; i < ctx->nptr; ++i)
+        if (!grads[i]) return DESLOC_E_NULL;
+
+    int dev_before = -1;
+    cudaError_t e = cudaGetDevice(&dev_before);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    if (dev_before != ctx->device) {
+        e = cudaSetDevice(ctx->device);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+    }
+    int rc = DESLOC_OK;
+    do {
+        void **d_g = nullptr;
+        rc = stage_grads(ctx, grads, stream, &d_g);
+        if (rc != DESLOC_OK) break;
+
+        // The mean of one replica is the replica: M = 1 always runs the local kernel.
+        const uint32_t kmask = (c.M == 1) ? 0u : mask;
+        const bool post = (c.flags & DESLOC_FLAG_POST_AVERAGE) != 0;
+        const void *fn = desloc::lookup_step_kernel(c.opt, post, c.grad_dtype == DESLOC_BF16,
+                                                    kmask ? c.M : 1, static_cast<int>(kmask));
+        if (!fn) {
+            rc = DESLOC_E_INVALID;
+            break;
+        }
+        desloc::StepArgs a{};
+        a.chunks = ctx->d_chunks;
+        a.nchunks = ctx->nchunks;
+        a.x = reinterpret_cast<float *const *>(ctx->d_tables);
+        a.u = reinterpret_cast<float *const *>(ctx->d_tables + ctx->nptr);
+        a.v = reinterpret_cast<float *const *>(ctx->d_tables + 2 * ctx->nptr);
+        a.g = reinterpret_cast<const void *const *>(d_g);
+        a.nt = c.num_tensors;
+        a.M = c.M;
+        a.b1 = c.beta1;
+        a.omb1 = static_cast<float>(1.0 - static_cast<double>(c.beta1));
+        a.b2 = c.beta2;
+        a.omb2 = static_cast<float>(1.0 - static_cast<double>(c.beta2));
+        a.eps = c.eps;
+        a.lam2 = static_cast<float>(static_cast<double>(c.eps) * static_cast<double>(c.eps));
+        a.lr = lr_t;
+        a.lrwd = static_cast<float>(static_cast<double>(lr_t) * static_cast<double>(c.weight_decay));
+        a.rho = c.clip_rho > 0.f ? c.clip_rho : std::numeric_limits<float>::infinity();
+        a.cbound = nclip ? clip_bound_t : std::numeric_limits<float>::infinity();
+
+        const long long nitems = kmask ? ctx->nchunks : ctx->nchunks * c.M;
+        long long grid = nitems;
+        if (ctx->ctas_per_sm > 0) {
+            const long long cap = static_cast<long long>(ctx->ctas_per_sm) * ctx->num_sms;
+            if (grid > cap) grid = cap;
+        }
+        if (grid > 0x7fffffffLL) grid = 0x7fffffffLL;  // the kernel strides over the rest
+        void *params[] = {&a};
+        e = cudaLaunchKernel(fn, dim3(static_cast<unsigned>(grid)), dim3(desloc::BLOCK_THREADS),
+                             params, 0, stream);
+        if (e != cudaSuccess) {
+            rc = cuda_fail(ctx, e);
+            break;
+        }
+        ctx->launches += 1;
+        Slot &s = ctx->slots[ctx->cur_slot];
+        e = cudaEventRecord(s.done, stream);
+        if (e != cudaSuccess) {
+            rc = cuda_fail(ctx, e);
+            break;
+        }
+        s.in_flight = true;
+        ctx->counters[0] += 1;
+        ctx->counters[1] += (mask & DESLOC_SYNC_X) ? 1 : 0;
+        ctx->counters[2] += (mask & DESLOC_SYNC_U) ? 1 : 0;
+        ctx->counters[3] += (mask & DESLOC_SYNC_V) ? 1 : 0;
+    } while (false);
+    if (dev_before != ctx->device) cudaSetDevice(dev_before);
+    return rc;
+}
+
+}  // namespace
+
+extern "C" {
+
+uint32_t desloc_sync_mask(const desloc_config *cfg, int64_t t) {
+    if (!cfg || t < 0) return 0;
+    return mask_at(cfg, t);
+}
+
+int64_t desloc_chunk_elems(void) { return desloc::CHUNK_ELEMS; }
+
+int64_t desloc_plan_chunks(const int64_t *numel, int32_t num_tensors, int64_t chunk_elems,
+                           int64_t *out, int64_t cap) {
+    if (!numel) return DESLOC_E_NULL;
+    if (num_tensors < 1 || chunk_elems < 1 || cap < 0) return DESLOC_E_RANGE;
+    if (cap > 0 && !out) return DESLOC_E_NULL;
+    int64_t n = 0;
+    for (int32_t k = 0; k < num_tensors; ++k) {
+        if (numel[k] < 1) return DESLOC_E_RANGE;
+        for (int64_t s = 0; s < numel[k]; s += chunk_elems) {
+            if (n < cap) {
+                out[3 * n + 0] = k;
+                out[3 * n + 1] = s;
+                out[3 * n + 2] = (numel[k] - s < chunk_elems) ? numel[k] - s : chunk_elems;
+            }
+            ++n;
+        }
+    }
+    return n;
+}
+
+int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *const *x, float *const *u,
+                  float *const *v, int cuda_device) {
+    if (!out) return DESLOC_E_NULL;
+    *out = nullptr;
+    int rc = validate_config(cfg);
+    if (rc != DESLOC_OK) return rc;
+    if (!cfg->numel || !x || !u) return DESLOC_E_NULL;
+    if (cfg->opt != DESLOC_SGDM && !v) return DESLOC_E_NULL;
+    if (cuda_device < 0) return DESLOC_E_RANGE;
+    const int64_t nptr = static_cast<int64_t>(cfg->M) * cfg->num_tensors;
+    int64_t total = 0;
+    for (int32_t k = 0; k < cfg->num_tensors; ++k) {
+        if (cfg->numel[k] < 1) return DESLOC_E_RANGE;
+        if (cfg->numel[k] > (INT64_MAX >> 4) - total) return DESLOC_E_RANGE;
+        total += cfg->numel[k];
+    }
+    for (int64_t i = 0; i < nptr; ++i) {
+        if (!x[i] || !u[i]) return DESLOC_E_NULL;
+        if (cfg->opt != DESLOC_SGDM && !v[i]) return DESLOC_E_NULL;
+    }
+
+    desloc_ctx *ctx = new (std::nothrow) desloc_ctx();
+    if (!ctx) return DESLOC_E_NOMEM;
+    std::vector<desloc::Chunk> chunks;
+    std::vector<void *> tables;
+    try {
+        ctx->numel.assign(cfg->numel, cfg->numel + cfg->num_tensors);
+        ctx->last_grads.assign(static_cast<size_t>(nptr), nullptr);
+        for (int32_t k = 0; k < cfg->num_tensors; ++k)
+            for (int64_t s = 0; s < cfg->numel[k]; s += desloc::CHUNK_ELEMS) {
+                desloc::Chunk ch;
+                ch.tensor = k;
+                ch.start = s;
+                const int64_t left = cfg->numel[k] - s;
+                ch.count = static_cast<int32_t>(left < desloc::CHUNK_ELEMS ? left : desloc::CHUNK_ELEMS);
+                chunks.push_back(ch);
+            }
+        tables.resize(static_cast<size_t>(3 * nptr), nullptr);
+        for (int64_t i = 0; i < nptr; ++i) {
+            tables[i] = x[i];
+            tables[nptr + i] = u[i];
+            tables[2 * nptr + i] = v ? static_cast<void *>(v[i]) : nullptr;
+        }
+    } catch (const std::bad_alloc &) {
+        delete ctx;
+        return DESLOC_E_NOMEM;
+    }
+    ctx->cfg = *cfg;
+    ctx->cfg.numel = ctx->numel.data();
+    ctx->device = cuda_device;
+    ctx->total_elems = total;
+    ctx->nptr = nptr;
+    ctx->nchunks = static_cast<int64_t>(chunks.size());
+
+    int dev_before = -1;
+    cudaError_t e = cudaGetDevice(&dev_before);
+    if (e == cudaSuccess && dev_before != cuda_device) e = cudaSetDevice(cuda_device);
+    if (e == cudaSuccess)
+        e = cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, cuda_device);
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_chunks, chunks.size() * sizeof(desloc::Chunk));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_tables, tables.size() * sizeof(void *));
+    if (e == cudaSuccess)
+        e = cudaMemcpy(ctx->d_chunks, chunks.data(), chunks.size() * sizeof(desloc::Chunk),
+                       cudaMemcpyHostToDevice);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(ctx->d_tables, tables.data(), tables.size() * sizeof(void *),
+                       cudaMemcpyHostToDevice);
+    for (int i = 0; i < kSlots && e == cudaSuccess; ++i) {
+        Slot &s = ctx->slots[i];
+        e = cudaMallocHost(&s.host, static_cast<size_t>(nptr) * sizeof(void *));
+        if (e == cudaSuccess) e = cudaMalloc(&s.dev, static_cast<size_t>(nptr) * sizeof(void *));
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming);
+    }
+    if (dev_before >= 0 && dev_before != cuda_device) cudaSetDevice(dev_before);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        free_ctx(ctx);
+        return e == cudaErrorMemoryAllocation ? DESLOC_E_NOMEM : DESLOC_E_CUDA;
+    }
+    *out = ctx;
+    return DESLOC_OK;
+}
+
+int desloc_step(desloc_ctx *ctx, int64_t t, float lr_t, float clip_bound_t,
+                const void *const *grads, void *stream, uint32_t *mask_out) {
+    if (!ctx || !grads) return DESLOC_E_NULL;
+    if (t < 0) return DESLOC_E_RANGE;
+    const uint32_t mask = mask_at(&ctx->cfg, t);
+    const int rc = run_step(ctx, mask, lr_t, clip_bound_t, grads, static_cast<cudaStream_t>(stream));
+    if (rc == DESLOC_OK && mask_out) *mask_out = mask;
+    return rc;
+}
+
+int desloc_step_masked(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
+                       const void *const *grads, void *stream) {
+    if (!ctx || !grads) return DESLOC_E_NULL;
+    if (mask & ~7u) return DESLOC_E_INVALID;
+    if (ctx->cfg.opt == DESLOC_SGDM && (mask & DESLOC_SYNC_V)) return DESLOC_E_INVALID;
+    return run_step(ctx, mask, lr_t, clip_bound_t, grads, static_cast<cudaStream_t>(stream));
+}
+
+int desloc_destroy(desloc_ctx *ctx) {
+    if (!ctx) return DESLOC_OK;
+    int dev_before = -1;
+    if (cudaGetDevice(&dev_before) == cudaSuccess && dev_before != ctx->device)
+        cudaSetDevice(ctx->device);
+    const int device = ctx->device;
+    free_ctx(ctx);
+    if (dev_before >= 0 && dev_before != device) cudaSetDevice(dev_before);
+    (void)cudaGetLastError();
+    return DESLOC_OK;
+}
+
+int desloc_get_counters(const desloc_ctx *ctx, int64_t out[4]) {
+    if (!ctx || !out) return DESLOC_E_NULL;
+    for (int i = 0; i < 4; ++i) out[i] = ctx->counters[i];
+    return DESLOC_OK;
+}
+
+int64_t desloc_get_launch_count(const desloc_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+int desloc_set_launch_shape(desloc_ctx *ctx, int32_t ctas_per_sm) {
+    if (!ctx) return DESLOC_E_NULL;
+    if (ctas_per_sm < 0 || ctas_per_sm > 32) return DESLOC_E_RANGE;
+    ctx->ctas_per_sm = ctas_per_sm;
+    return DESLOC_OK;
+}
+
+int desloc_last_cuda_error(const desloc_ctx *ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+const char *desloc_strerror(int status) {
+    switch (status) {
+        case DESLOC_OK: return "ok";
+        case DESLOC_E_NULL: return "a required pointer is NULL";
+        case DESLOC_E_RANGE: return "argument out of range";
+        case DESLOC_E_INVALID: return "invalid optimizer, dtype, flag or mask";
+        case DESLOC_E_NOMEM: return "out of memory";
+        case DESLOC_E_CUDA: return "CUDA call failed";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

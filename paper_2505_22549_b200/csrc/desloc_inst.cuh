@@ -1,0 +1,44 @@
+// Instantiation tables for desloc_step_kernel.  Each optimizer x averaging order is its own
+// translation unit (they compile in parallel); this header builds the (MT, mask) -> kernel
+// table for one of them.
+#pragma once
+#include <utility>
+
+#include "desloc_kernels.cuh"
+
+namespace desloc {
+
+template <int OPT, bool POST, typename GT, int MT, int MASK>
+const void *kernel_ptr() {
+    return reinterpret_cast<const void *>(&desloc_step_kernel<OPT, MASK, MT, GT, POST>);
+}
+
+// NMASK = 7 (masks 1..7) for Adam / ADOPT, 3 (masks 1..3: no second state) for SGDM.
+template <int OPT, bool POST, typename GT, int NMASK, int... I>
+const void *pick_sync(int mt, int mask, std::integer_sequence<int, I...>) {
+    static const void *const tbl[] = {kernel_ptr<OPT, POST, GT, 2 + I / NMASK, 1 + I % NMASK>()...};
+    if (mt < 2 || mt > MAX_MT || mask < 1 || mask > NMASK) return nullptr;
+    return tbl[(mt - 2) * NMASK + (mask - 1)];
+}
+
+template <int OPT, bool POST>
+const void *lookup_sync(bool bf16, int mt, int mask) {
+    constexpr int NMASK = (OPT == OPT_SGDM) ? 3 : 7;
+    using Seq = std::make_integer_sequence<int, (MAX_MT - 1) * NMASK>;
+    return bf16 ? pick_sync<OPT, POST, bf16_t, NMASK>(mt, mask, Seq{})
+                : pick_sync<OPT, POST, float, NMASK>(mt, mask, Seq{});
+}
+
+template <int OPT>
+const void *lookup_local(bool bf16) {
+    return bf16 ? kernel_ptr<OPT, false, bf16_t, 1, 0>() : kernel_ptr<OPT, false, float, 1, 0>();
+}
+
+const void *lookup_adam_pre(bool bf16, int mt, int mask);
+const void *lookup_adam_post(bool bf16, int mt, int mask);
+const void *lookup_adopt_pre(bool bf16, int mt, int mask);
+const void *lookup_adopt_post(bool bf16, int mt, int mask);
+const void *lookup_sgdm_pre(bool bf16, int mt, int mask);
+const void *lookup_sgdm_post(bool bf16, int mt, int mask);
+
+}  // namespace desloc

@@ -1,0 +1,298 @@
+// DES-LOC fused step kernel for sm_100a: one streaming pass over g, x, u, v of all M
+// worker replicas (Algorithm 1 with the Adam, ADOPT and SGDM rules of Algorithms 2-3).
+//
+// Work decomposition.  The tensor list is cut into chunks of CHUNK_ELEMS elements of one
+// tensor (table built once on the host).  A thread block takes one chunk at a time:
+//   * local steps (no array synced) treat workers independently: the work item is
+//     (worker, chunk) and the kernel is the MT = 1 instantiation;
+//   * sync steps are instantiated per worker count MT = M and per sync mask: a thread loads
+//     its elements of all M replicas, sums the synced arrays in the fixed order m = 0..M-1,
+//     and writes every replica back -- the same bytes as a local step.
+// Every thread issues all loads of its tile (MT workers x UN positions x 4 arrays, 128-bit
+// where aligned) before the first use, so that enough bytes are in flight to cover HBM
+// latency; the arithmetic is fp32.  Tensors whose pointers are not 16-byte aligned and the
+// last (numel mod 4) elements of a tensor take the scalar instantiation of the same code.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace desloc {
+
+constexpr int OPT_ADAM = 0, OPT_ADOPT = 1, OPT_SGDM = 2;
+constexpr int SYNC_X = 1, SYNC_U = 2, SYNC_V = 4;
+constexpr int BLOCK_THREADS = 256;
+constexpr int CHUNK_ELEMS = 4096;  // 256 threads x 4 elements x 4 positions
+constexpr int MAX_MT = 8;          // largest worker count with a register-resident kernel
+
+struct __align__(16) Chunk {
+    int32_t tensor;  // index into the tensor list
+    int32_t count;   // elements in this chunk (<= CHUNK_ELEMS)
+    int64_t start;   // first element within the tensor
+};
+
+struct StepArgs {
+    const Chunk *chunks;
+    long long nchunks;
+    float *const *x;  // device tables [M * nt], entry m * nt + k
+    float *const *u;
+    float *const *v;
+    const void *const *g;
+    int nt;
+    int M;
+    float b1, omb1;   // beta1, 1 - beta1
+    float b2, omb2;   // beta2, 1 - beta2
+    float eps;        // ADOPT epsilon
+    float lam2;       // Adam lambda^2
+    float lr;         // eta_t
+    float lrwd;       // eta_t * weight_decay
+    float rho;        // coordinate clip radius, +inf when off
+    float cbound;     // ADOPT normalised-gradient bound, +inf when off
+};
+
+struct bf16_t {
+    uint16_t bits;
+};
+
+template <int VEC>
+struct FV {
+    float a[VEC];
+};
+
+// ---- global memory access: streaming (evict-first) 128-bit or scalar ---------------------
+template <int VEC>
+__device__ __forceinline__ FV<VEC> ld_f32(const char *base, long long elem) {
+    FV<VEC> r;
+    if constexpr (VEC == 4) {
+        const float4 t = __ldcs(reinterpret_cast<const float4 *>(base) + (elem >> 2));
+        r.a[0] = t.x; r.a[1] = t.y; r.a[2] = t.z; r.a[3] = t.w;
+    } else {
+        r.a[0] = __ldcs(reinterpret_cast<const float *>(base) + elem);
+    }
+    return r;
+}
+
+template <int VEC>
+__device__ __forceinline__ void st_f32(char *base, long long elem, const FV<VEC> &r) {
+    if constexpr (VEC == 4) {
+        __stcs(reinterpret_cast<float4 *>(base) + (elem >> 2),
+               make_float4(r.a[0], r.a[1], r.a[2], r.a[3]));
+    } else {
+        __stcs(reinterpret_cast<float *>(base) + elem, r.a[0]);
+    }
+}
+
+template <int VEC, typename GT>
+__device__ __forceinline__ FV<VEC> ld_grad(const char *base, long long elem) {
+    FV<VEC> r;
+    if constexpr (sizeof(GT) == 4) {
+        r = ld_f32<VEC>(base, elem);
+    } else if constexpr (VEC == 4) {
+        // four bf16 in 8 bytes; bf16 -> fp32 is a 16-bit shift (exact)
+        const uint2 t = __ldcs(reinterpret_cast<const uint2 *>(base) + (elem >> 2));
+        r.a[0] = __uint_as_float(t.x << 16);
+        r.a[1] = __uint_as_float(t.x & 0xffff0000u);
+        r.a[2] = __uint_as_float(t.y << 16);
+        r.a[3] = __uint_as_float(t.y & 0xffff0000u);
+    } else {
+        const unsigned short t = __ldcs(reinterpret_cast<const unsigned short *>(base) + elem);
+        r.a[0] = __uint_as_float(static_cast<unsigned>(t) << 16);
+    }
+    return r;
+}
+
+// ---- the update of one coordinate across all MT workers (registers only) -----------------
+// Pre-average (Algorithms 1-3): synced arrays are replaced by their worker mean BEFORE the
+// update.  Post-average (Algorithms 4-5): the updated values are averaged, and the parameter
+// step uses the averaged states.  Sums run m = 0..MT-1 in that order.
+template <int MT>
+__device__ __forceinline__ float mean_of(const float (&s)[MT]) {
+    float acc = s[0];
+#pragma unroll
+    for (int m = 1; m < MT; ++m) acc += s[m];
+    return acc / static_cast<float>(MT);
+}
+
+template <int OPT, int MASK, int MT, bool POST>
+__device__ __forceinline__ void update_coord(const StepArgs &a, const float (&g)[MT],
+                                             float (&x)[MT], float (&u)[MT], float (&v)[MT]) {
+    constexpr bool PRE = !POST;
+    float xb = 0.f, ub = 0.f, vb = 0.f;
+    if constexpr (PRE && (MASK & SYNC_X)) xb = mean_of<MT>(x);
+    if constexpr (PRE && (MASK & SYNC_U)) ub = mean_of<MT>(u);
+    if constexpr (PRE && (MASK & SYNC_V) && OPT != OPT_SGDM) vb = mean_of<MT>(v);
+
+    float un[MT], vn[MT], xn[MT];
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+        // coordinate-wise clip: sgn(g) min(|g|, rho)  (Section 3.1); rho = +inf when off
+        const float gh = fminf(fmaxf(g[m], -a.rho), a.rho);
+        const float up = (PRE && (MASK & SYNC_U)) ? ub : u[m];
+        if constexpr (OPT == OPT_ADAM) {
+            const float vp = (PRE && (MASK & SYNC_V)) ? vb : v[m];
+            un[m] = fmaf(a.b1, up, a.omb1 * gh);
+            vn[m] = fmaf(a.b2, vp, (a.omb2 * gh) * gh);
+        } else if constexpr (OPT == OPT_ADOPT) {
+            const float vp = (PRE && (MASK & SYNC_V)) ? vb : v[m];
+            vn[m] = fmaf(a.b2, vp, (a.omb2 * gh) * gh);
+            // normalised by the worker's own v from before this step
+            float r = gh / fmaxf(sqrtf(v[m]), a.eps);
+            r = fminf(fmaxf(r, -a.cbound), a.cbound);
+            un[m] = fmaf(a.b1, up, a.omb1 * r);
+        } else {
+            un[m] = fmaf(a.b1, up, a.omb1 * gh);
+            vn[m] = 0.f;
+        }
+    }
+    if constexpr (POST && (MASK & SYNC_U)) {
+        const float mu = mean_of<MT>(un);
+#pragma unroll
+        for (int m = 0; m < MT; ++m) un[m] = mu;
+    }
+    if constexpr (POST && (MASK & SYNC_V) && OPT != OPT_SGDM) {
+        const float mv = mean_of<MT>(vn);
+#pragma unroll
+        for (int m = 0; m < MT; ++m) vn[m] = mv;
+    }
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+        const float xp = (PRE && (MASK & SYNC_X)) ? xb : x[m];
+        float d;
+        if constexpr (OPT == OPT_ADAM)
+            d = (a.lr * un[m]) / sqrtf(vn[m] + a.lam2);
+        else
+            d = a.lr * un[m];
+        // x* (1 - eta wd) - d, written as x* - (eta wd x* + d): one rounding at x's scale
+        xn[m] = xp - fmaf(a.lrwd, xp, d);
+    }
+    if constexpr (POST && (MASK & SYNC_X)) {
+        const float mx = mean_of<MT>(xn);
+#pragma unroll
+        for (int m = 0; m < MT; ++m) xn[m] = mx;
+    }
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+        x[m] = xn[m];
+        u[m] = un[m];
+        v[m] = vn[m];
+    }
+}
+
+// ---- one thread's tile: MT workers x UN positions of VEC elements ------------------------
+// sp[arr][m] are chunk-relative base pointers in shared memory (arr: 0 x, 1 u, 2 v, 3 g).
+// Position j covers elements e0 + j * pstride .. + VEC - 1; positions >= npos are skipped.
+template <int OPT, int MASK, int MT, typename GT, bool POST, int VEC, int UN, bool FULL>
+__device__ __forceinline__ void process_tile(const StepArgs &a, char *const (*sp)[MT],
+                                             long long e0, int pstride, int npos) {
+    FV<VEC> G[UN][MT], X[UN][MT], U[UN][MT], V[UN][MT];
+#pragma unroll
+    for (int j = 0; j < UN; ++j) {
+        if (FULL || j < npos) {
+            const long long e = e0 + static_cast<long long>(j) * pstride;
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                G[j][m] = ld_grad<VEC, GT>(sp[3][m], e);
+                X[j][m] = ld_f32<VEC>(sp[0][m], e);
+                U[j][m] = ld_f32<VEC>(sp[1][m], e);
+                if constexpr (OPT != OPT_SGDM) V[j][m] = ld_f32<VEC>(sp[2][m], e);
+            }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < UN; ++j) {
+        if (FULL || j < npos) {
+            const long long e = e0 + static_cast<long long>(j) * pstride;
+#pragma unroll
+            for (int c = 0; c < VEC; ++c) {
+                float g[MT], x[MT], u[MT], v[MT];
+#pragma unroll
+                for (int m = 0; m < MT; ++m) {
+                    g[m] = G[j][m].a[c];
+                    x[m] = X[j][m].a[c];
+                    u[m] = U[j][m].a[c];
+                    v[m] = (OPT != OPT_SGDM) ? V[j][m].a[c] : 0.f;
+                }
+                update_coord<OPT, MASK, MT, POST>(a, g, x, u, v);
+#pragma unroll
+                for (int m = 0; m < MT; ++m) {
+                    X[j][m].a[c] = x[m];
+                    U[j][m].a[c] = u[m];
+                    if constexpr (OPT != OPT_SGDM) V[j][m].a[c] = v[m];
+                }
+            }
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                st_f32<VEC>(sp[0][m], e, X[j][m]);
+                st_f32<VEC>(sp[1][m], e, U[j][m]);
+                if constexpr (OPT != OPT_SGDM) st_f32<VEC>(sp[2][m], e, V[j][m]);
+            }
+        }
+    }
+}
+
+template <int MT>
+struct UnrollFor {
+    static constexpr int value = MT == 1 ? 4 : (MT == 2 ? 2 : 1);
+};
+
+template <int OPT, int MASK, int MT, typename GT, bool POST>
+__global__ void __launch_bounds__(BLOCK_THREADS, (MT <= 4 ? 3 : 2))
+desloc_step_kernel(const __grid_constant__ StepArgs a) {
+    constexpr int UN = UnrollFor<MT>::value;
+    __shared__ char *sp[4][MT];
+    const int tid = threadIdx.x;
+    // MT == 1 serves local steps of any M: item = (worker, chunk), workers independent.
+    const long long nitems = (MT == 1) ? a.nchunks * a.M : a.nchunks;
+    for (long long item = blockIdx.x; item < nitems; item += gridDim.x) {
+        const long long c = (MT == 1) ? item % a.nchunks : item;
+        const int m0 = (MT == 1) ? static_cast<int>(item / a.nchunks) : 0;
+        const Chunk ch = a.chunks[c];
+        __syncthreads();  // previous chunk's readers are done with sp
+        int misaligned = 0;
+        if (tid < 4 * MT) {
+            const int arr = tid / MT, m = tid - arr * MT;
+            const long long idx = static_cast<long long>(m0 + m) * a.nt + ch.tensor;
+            char *p = nullptr;
+            if (arr == 0) p = reinterpret_cast<char *>(a.x[idx]) + ch.start * 4;
+            if (arr == 1) p = reinterpret_cast<char *>(a.u[idx]) + ch.start * 4;
+            if (arr == 2 && OPT != OPT_SGDM) p = reinterpret_cast<char *>(a.v[idx]) + ch.start * 4;
+            if (arr == 3)
+                p = const_cast<char *>(reinterpret_cast<const char *>(a.g[idx])) +
+                    ch.start * static_cast<long long>(sizeof(GT));
+            sp[arr][m] = p;
+            const unsigned need = (arr == 3 && sizeof(GT) == 2) ? 7u : 15u;
+            misaligned = (reinterpret_cast<uintptr_t>(p) & need) != 0;
+        }
+        const int scalar_path = __syncthreads_or(misaligned);
+        if (!scalar_path) {
+            if (ch.count == CHUNK_ELEMS) {
+                // full chunk: 4 * UN * 256 * (4 / UN) elements, no bounds checks
+#pragma unroll 1
+                for (int r = 0; r < 4 / UN; ++r)
+                    process_tile<OPT, MASK, MT, GT, POST, 4, UN, true>(
+                        a, sp, static_cast<long long>(r * UN * BLOCK_THREADS + tid) * 4,
+                        BLOCK_THREADS * 4, UN);
+            } else {
+                const int n4 = ch.count >> 2;
+                for (int p0 = tid; p0 < n4; p0 += UN * BLOCK_THREADS) {
+                    const int left = (n4 - p0 + BLOCK_THREADS - 1) / BLOCK_THREADS;
+                    process_tile<OPT, MASK, MT, GT, POST, 4, UN, false>(
+                        a, sp, static_cast<long long>(p0) * 4, BLOCK_THREADS * 4,
+                        left < UN ? left : UN);
+                }
+                const int rem = ch.count & 3;
+                if (tid < rem)
+                    process_tile<OPT, MASK, MT, GT, POST, 1, 1, true>(a, sp, (n4 << 2) + tid, 0, 1);
+            }
+        } else {
+            for (int e = tid; e < ch.count; e += BLOCK_THREADS)
+                process_tile<OPT, MASK, MT, GT, POST, 1, 1, true>(a, sp, e, 0, 1);
+        }
+    }
+}
+
+// Lookup of an instantiation: opt, post-average?, bf16 gradients?, MT in 1..MAX_MT, mask.
+// MT == 1 exists only with mask 0 (the mean of one replica is itself).  Returns nullptr for
+// combinations that do not exist.
+const void *lookup_step_kernel(int opt, bool post, bool bf16, int mt, int mask);
+
+}  // namespace desloc

@@ -1,0 +1,89 @@
+"""``DesLoc``: owns nothing but a context handle; holds references to the caller's tensors."""
+from __future__ import annotations
+
+from typing import List, Optional, Sequence
+
+import torch
+
+from . import binding as B
+
+
+class DesLoc:
+    """M worker replicas of a tensor list, stepped by the CUDA library.
+
+    x, u, v: lists (one per worker) of lists of CUDA fp32 tensors (one per model tensor),
+    updated in place by :meth:`step`.  v is None for SGDM.
+    """
+
+    def __init__(self, x: Sequence[Sequence[torch.Tensor]], u, v, *, opt, grad_dtype,
+                 beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0, clip_rho=0.0,
+                 K=(1, 1, 1), flags=0):
+        M = len(x)
+        numel = [int(t.numel()) for t in x[0]]
+        dev = x[0][0].device
+        if dev.type != "cuda":
+            raise ValueError("DesLoc needs CUDA tensors (there is no CPU path)")
+        for arrs in (x, u) + ((v,) if v is not None else ()):
+            if len(arrs) != M:
+                raise ValueError("x, u, v need one tensor list per worker")
+            for lst in arrs:
+                if [int(t.numel()) for t in lst] != numel:
+                    raise ValueError("every worker needs the same tensor list")
+                for t in lst:
+                    if t.dtype != torch.float32 or not t.is_contiguous() or t.device != dev:
+                        raise ValueError("state tensors must be contiguous fp32 on one device")
+        self._keep = (x, u, v)
+        self.M, self.numel, self.device = M, numel, dev
+        self.grad_dtype = B.DTYPE_BY_NAME.get(grad_dtype, grad_dtype)
+        self.cfg = B.make_config(M, numel, opt, grad_dtype, beta1, beta2, eps, weight_decay,
+                                 clip_rho, K[0], K[1], K[2], flags)
+        flat = lambda a: [t.data_ptr() for lst in a for t in lst]
+        self.ctx: Optional[int] = B.desloc_create(
+            self.cfg, flat(x), flat(u), flat(v) if v is not None else None,
+            dev.index if dev.index is not None else torch.cuda.current_device())
+        self._gkey = None
+        self._garr = None
+
+    def _grad_array(self, grads: Sequence[Sequence[torch.Tensor]]):
+        want = torch.bfloat16 if self.grad_dtype == B.DESLOC_BF16 else torch.float32
+        ptrs: List[int] = []
+        for lst in grads:
+            for t, n in zip(lst, self.numel):
+                if t.dtype != want or t.numel() != n or not t.is_contiguous():
+                    raise ValueError("gradient tensor of wrong dtype, size or layout")
+                ptrs.append(t.data_ptr())
+        if len(ptrs) != self.M * len(self.numel):
+            raise ValueError("need one gradient list per worker")
+        key = tuple(ptrs)
+        if key != self._gkey:
+            self._gkey, self._garr = key, B.ptr_array(ptrs)
+        return self._garr
+
+    def step(self, t: int, lr: float, grads, clip_bound: float = 0.0) -> int:
+        """Step t on torch's current stream; returns the sync mask."""
+        stream = torch.cuda.current_stream(self.device).cuda_stream
+        return B.desloc_step(self.ctx, t, lr, clip_bound, self._grad_array(grads), stream)
+
+    def step_masked(self, mask: int, lr: float, grads, clip_bound: float = 0.0) -> None:
+        stream = torch.cuda.current_stream(self.device).cuda_stream
+        B.desloc_step_masked(self.ctx, mask, lr, clip_bound, self._grad_array(grads), stream)
+
+    def counters(self):
+        return B.desloc_get_counters(self.ctx)
+
+    def launches(self) -> int:
+        return B.desloc_get_launch_count(self.ctx)
+
+    def set_launch_shape(self, ctas_per_sm: int) -> None:
+        B.desloc_set_launch_shape(self.ctx, ctas_per_sm)
+
+    def close(self) -> None:
+        if self.ctx is not None:
+            B.desloc_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,127 @@
+"""Host-side checks that need no GPU: the shared library loads and exports every symbol the
+header declares, the schedule and the chunk plan are right, and bad arguments are rejected
+before any CUDA call."""
+import os
+import re
+
+import pytest
+
+import desloc_inputs as di
+import oracle
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def d():
+    from paper_2505_22549_b200 import build
+    build.build()
+    import paper_2505_22549_b200 as lib
+    return lib
+
+
+def test_library_exports_every_declared_symbol(d):
+    header = open(os.path.join(ROOT, "include", "desloc.h")).read()
+    names = re.findall(r"DESLOC_API\s+[\w\s\*]+?\b(desloc_\w+)\s*\(", header)
+    assert len(names) >= 12 and len(set(names)) == len(names)
+    L = d.raw_lib()
+    for n in names:
+        assert hasattr(L, n), f"{n} declared in desloc.h but not exported"
+
+
+def test_sync_mask_matches_oracle_schedule(d):
+    for opt, oid in (("adam", oracle.ADAM), ("adopt", oracle.ADOPT), ("sgdm", oracle.SGDM)):
+        for K in [(4, 8, 16), (1, 1, 1), (16, 64, 256), (0, 0, 0), (3, 0, 7), (256, 768, 1536)]:
+            cfg = d.make_config(2, [8], opt, "bf16", Kx=K[0], Ku=K[1], Kv=K[2])
+            for t in list(range(0, 70)) + [255, 256, 767, 768, 1536, 3072, 2 ** 40]:
+                assert d.desloc_sync_mask(cfg, t) == oracle.sync_mask(oid, K[0], K[1], K[2], t)
+    assert d.desloc_sync_mask(None, 0) == 0
+    cfg = d.make_config(2, [8], "adam", "bf16")
+    assert d.desloc_sync_mask(cfg, -1) == 0
+
+
+def test_chunk_plan_covers_every_element_once(d):
+    ce = d.desloc_chunk_elems()
+    assert ce == 4096
+    for numel in [[1], [ce], [ce + 1], [3, ce * 2, 5, ce * 3 - 1], list(di.mini(di.WORKLOADS["cfg2_adam_135m"]).numel)]:
+        total, chunks = d.desloc_plan_chunks(numel, ce)
+        assert total == len(chunks) == sum(-(-n // ce) for n in numel)
+        seen = [0] * len(numel)
+        for k, s, c in chunks:
+            assert s == seen[k] and 1 <= c <= ce
+            assert c == ce or s + c == numel[k]      # only a tensor's last chunk is short
+            seen[k] += c
+        assert seen == list(numel)
+    # capacity smaller than needed: still reports the full count
+    total, chunks = d.desloc_plan_chunks([ce * 10], ce, cap=3)
+    assert total == 10 and len(chunks) == 3
+    # full-size list of the 1.7B workload
+    w = di.WORKLOADS["cfg4_adam_1p7b"]
+    total, _ = d.desloc_plan_chunks(w.numel, ce, cap=0)
+    assert total == sum(-(-n // ce) for n in w.numel)
+    with pytest.raises(d.DeslocError) as e:
+        d.desloc_plan_chunks([5, 0], ce)
+    assert e.value.status == d.DESLOC_E_RANGE
+
+
+def test_workload_sizes_match_the_stated_totals():
+    assert di.WORKLOADS["cfg2_adam_135m"].N == 134_515_008
+    assert di.WORKLOADS["cfg3_adopt_360m"].N == 361_821_120
+    assert di.WORKLOADS["cfg4_adam_1p7b"].N == 1_711_376_384
+    assert len(di.WORKLOADS["cfg4_adam_1p7b"].numel) == 218
+
+
+BAD = [
+    (dict(M=0), "DESLOC_E_RANGE"), (dict(M=65), "DESLOC_E_RANGE"),
+    (dict(Kx=-1), "DESLOC_E_RANGE"), (dict(beta1=1.0), "DESLOC_E_RANGE"),
+    (dict(beta2=-0.1), "DESLOC_E_RANGE"), (dict(beta1=float("nan")), "DESLOC_E_RANGE"),
+    (dict(eps=-1.0), "DESLOC_E_RANGE"), (dict(weight_decay=-1.0), "DESLOC_E_RANGE"),
+    (dict(opt=3), "DESLOC_E_INVALID"), (dict(grad_dtype=2), "DESLOC_E_INVALID"),
+    (dict(flags=4), "DESLOC_E_INVALID"), (dict(flags=1), "DESLOC_E_INVALID"),  # norm clip w/o ADOPT
+    (dict(numel=[4, 0]), "DESLOC_E_RANGE"),
+]
+
+
+@pytest.mark.parametrize("kw,status", BAD)
+def test_create_rejects_bad_config_before_touching_the_device(d, kw, status):
+    args = dict(M=2, numel=[4, 4], opt="adam", grad_dtype="f32")
+    args.update(kw)
+    cfg = d.make_config(**args)
+    n = max(1, cfg.M) * len(args["numel"])
+    with pytest.raises(d.DeslocError) as e:
+        d.desloc_create(cfg, [16] * n, [16] * n, [16] * n, 0)
+    assert e.value.status == getattr(d, status)
+
+
+def test_create_rejects_null_pointers(d):
+    cfg = d.make_config(2, [4], "adam", "f32")
+    for x, u, v in [([16, 0], [16, 16], [16, 16]), ([16, 16], None, [16, 16]),
+                    ([16, 16], [16, 16], None), ([16, 16], [16, 16], [0, 16])]:
+        with pytest.raises(d.DeslocError) as e:
+            d.desloc_create(cfg, x, u, v, 0)
+        assert e.value.status == d.DESLOC_E_NULL
+    # SGDM needs no v
+    cfg = d.make_config(2, [4], "sgdm", "f32")
+    with pytest.raises(d.DeslocError) as e:
+        d.desloc_create(cfg, [16, 16], [16, 16], None, -1)
+    assert e.value.status == d.DESLOC_E_RANGE
+
+
+def test_null_context_is_handled(d):
+    L = d.raw_lib()
+    assert L.desloc_destroy(None) == 0
+    assert L.desloc_step(None, 0, 0.1, 0.0, None, None, None) == d.DESLOC_E_NULL
+    assert L.desloc_get_counters(None, None) == d.DESLOC_E_NULL
+    assert L.desloc_get_launch_count(None) == 0
+    assert d.desloc_strerror(0) == "ok" and "unknown" in d.desloc_strerror(-99)
+
+
+def test_no_cpu_fallback_without_a_device(d):
+    """On a machine without a GPU a valid create must fail with a CUDA status, not fall back."""
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    cfg = d.make_config(1, [4], "adam", "f32")
+    with pytest.raises(d.DeslocError) as e:
+        d.desloc_create(cfg, [16], [16], [16], 0)
+    assert e.value.status in (d.DESLOC_E_CUDA, d.DESLOC_E_NOMEM)

@@ -1,0 +1,261 @@
+"""GPU parity: the CUDA library (through its C ABI binding) against the CPU oracle, element by
+element on the same seeded inputs.  Bar: relative error <= 1e-5 on fp32 x, u, v after T steps
+(denominator max(|ref|, rms(ref tensor))), sync masks and counters exact as integers."""
+import numpy as np
+import pytest
+import torch
+
+import desloc_inputs as di
+import oracle
+from _util import OPT_ID, TOL, State, compare_per_tensor, f32r, oracle_cfg, rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+def _lib():
+    import paper_2505_22549_b200 as d
+    return d
+
+
+def _flags(d, w, post=False):
+    f = 0
+    if w.adopt_norm_clip:
+        f |= d.DESLOC_FLAG_ADOPT_NORM_CLIP
+    if post:
+        f |= d.DESLOC_FLAG_POST_AVERAGE
+    return f
+
+
+def make_engine(d, w, st, post=False):
+    return d.DesLoc(st.views(st.x), st.views(st.u), st.views(st.v) if st.v is not None else None,
+                    opt=w.opt, grad_dtype=w.grad_dtype, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
+                    weight_decay=w.weight_decay, clip_rho=w.clip_rho, K=w.K,
+                    flags=_flags(d, w, post))
+
+
+def run_both(w, T, align=4, byte_shift=0, post=False, v_init=0.0, identical=False,
+             forced_masks=None, lr_of_t=None, ctas_per_sm=0):
+    """Runs T steps on the GPU and in the oracle on identical inputs; returns both end states."""
+    d = _lib()
+    dev = torch.device("cuda:0")
+    st = State(w, dev, align=align, byte_shift=byte_shift, v_init=v_init)
+    eng = make_engine(d, w, st, post)
+    if ctas_per_sm:
+        eng.set_launch_shape(ctas_per_sm)
+    ox, ou = st.to_numpy(st.x), st.to_numpy(st.u)
+    ov = st.to_numpy(st.v) if st.v is not None else None
+    ocfg = oracle_cfg(w, oracle.FLAG_POST_AVERAGE if post else 0)
+    gviews = st.views(st.g)
+    gpu_masks, ref_masks = [], []
+    for t in range(T):
+        st.fill_grads(t, identical=identical)
+        lr = f32r(lr_of_t(t) if lr_of_t else w.lr)
+        cb = f32r(w.clip_bound(t))
+        g_host = st.to_numpy(st.g)
+        if forced_masks is None:
+            gpu_masks.append(eng.step(t, lr, gviews, clip_bound=cb))
+            ref_masks.append(oracle.step(ocfg, t, lr, ox, ou, ov, g_host, clip_bound=cb))
+        else:
+            # force one sync pattern: the oracle gets periods that produce it at t = 0, else none
+            mk = forced_masks[t]
+            eng.step_masked(mk, lr, gviews, clip_bound=cb)
+            c2 = oracle_cfg(w.replace(K=(mk & 1, (mk >> 1) & 1, (mk >> 2) & 1)),
+                            oracle.FLAG_POST_AVERAGE if post else 0)
+            got = oracle.step(c2, 0, lr, ox, ou, ov, g_host, clip_bound=cb)
+            assert got == mk
+    torch.cuda.synchronize()
+    res = dict(st=st, gx=st.to_numpy(st.x), gu=st.to_numpy(st.u),
+               gv=st.to_numpy(st.v) if st.v is not None else None, ox=ox, ou=ou, ov=ov,
+               gpu_masks=gpu_masks, ref_masks=ref_masks, counters=eng.counters(),
+               launches=eng.launches())
+    eng.close()
+    return res
+
+
+def check(res, tol=TOL):
+    st = res["st"]
+    worst = {"x": compare_per_tensor(st, res["gx"], res["ox"], "x", tol),
+             "u": compare_per_tensor(st, res["gu"], res["ou"], "u", tol)}
+    if res["gv"] is not None:
+        worst["v"] = compare_per_tensor(st, res["gv"], res["ov"], "v", tol)
+    assert res["gpu_masks"] == res["ref_masks"]
+    return worst
+
+
+# ------------------------------------------------------------------ config 1, all elements
+def test_cfg1_adam_n4096_full_run():
+    w = di.WORKLOADS["cfg1_adam_n4096"]
+    res = run_both(w, w.T)
+    check(res)
+    assert res["gpu_masks"][:9] == [7, 0, 0, 0, 1, 0, 0, 0, 3]
+    assert res["counters"] == [64, 16, 8, 4]
+    assert res["launches"] == 64            # one kernel per step
+    # the run really moved the parameters (the check is not vacuous)
+    x0 = di.init_params(w).numpy()
+    assert np.max(np.abs(res["gx"][0] - x0)) > 1e-2
+
+
+# ------------------------------------------------------------------ tiny and ragged shapes
+@pytest.mark.parametrize("opt", ["adam", "adopt", "sgdm"])
+@pytest.mark.parametrize("M", [1, 2, 3, 4, 5, 6, 7, 8])
+@pytest.mark.parametrize("gd", ["f32", "bf16"])
+def test_every_mask_on_ragged_tensors(opt, M, gd):
+    """Tensors of 1..9 elements, one chunk + 1, odd sizes; all 8 sync patterns in turn, twice."""
+    numel = (1, 2, 3, 4, 5, 7, 8, 9, 4095, 4096, 4097, 8191, 12289, 31)
+    nmask = 4 if opt == "sgdm" else 8
+    masks = list(range(nmask)) * 2
+    w = di.Workload(f"tiny_{opt}", opt, M, numel, gd, "normal1", beta1=0.9, beta2=0.99,
+                    eps=1e-3 if opt != "adopt" else 1e-2, lr=1e-2, weight_decay=0.05,
+                    clip_rho=1.5, adopt_norm_clip=(opt == "adopt"), seed=M)
+    for align in (4, 1):   # 4: vector path with tails; 1: packed, odd offsets -> scalar path
+        res = run_both(w, len(masks), align=align, forced_masks=masks, v_init=0.25)
+        check(res)
+
+
+@pytest.mark.parametrize("opt", ["adam", "adopt", "sgdm"])
+@pytest.mark.parametrize("M", [2, 3, 8])
+def test_post_average_ordering(opt, M):
+    numel = (5, 4096, 4099, 1000)
+    nmask = 4 if opt == "sgdm" else 8
+    masks = list(range(nmask)) + [nmask - 1]
+    w = di.Workload(f"post_{opt}", opt, M, numel, "bf16", "normal1", beta1=0.9, beta2=0.99,
+                    eps=1e-2, lr=1e-2, clip_rho=2.0, seed=7 + M)
+    res = run_both(w, len(masks), forced_masks=masks, post=True, v_init=0.5)
+    check(res)
+    # after a step that averaged everything, replicas are bitwise equal
+    for a in ("gx", "gu") + (("gv",) if opt != "sgdm" else ()):
+        for m in range(1, M):
+            assert np.array_equal(res[a][0], res[a][m])
+
+
+def test_misaligned_buffers_take_the_scalar_path():
+    w = di.Workload("shift", "adam", 3, (4096 * 2 + 5, 17), "bf16", "normal1", lr=1e-2,
+                    K=(2, 3, 4), seed=3)
+    for shift in (1, 2, 3):
+        res = run_both(w, 6, align=1, byte_shift=shift)
+        check(res)
+
+
+# ------------------------------------------------------------------ scaled-down paper workloads
+MINI = ["cfg2_adam_135m", "cfg3_adopt_360m", "cfg4_adam_1p7b", "cfg5_sgdm_ddp", "cfg5_sgdm_desloc",
+        "cfg5_adam_local", "cfg5_adam_desloc"]
+
+
+@pytest.mark.parametrize("name", MINI)
+def test_mini_workloads_full_oracle(name):
+    """Same recipe (optimizer, M, gradient distribution, hyper-parameters) on a 2-layer model
+    of 21 tensors; periods shortened so that T = 40 steps see every sync pattern."""
+    w = di.mini(di.WORKLOADS[name], T=40)
+    if max(w.K) > 16:
+        w = w.replace(K=tuple(max(1, k // 8) for k in w.K))
+    res = run_both(w, w.T, ctas_per_sm=0)
+    worst = check(res)
+    assert res["counters"][0] == w.T
+    assert sum(res["counters"][1:]) == sum(bin(m).count("1") for m in res["ref_masks"])
+    print(name, worst)
+
+
+def test_persistent_grid_gives_identical_bits():
+    w = di.mini(di.WORKLOADS["cfg2_adam_135m"], T=12).replace(K=(2, 3, 4))
+    a = run_both(w, w.T, ctas_per_sm=0)
+    b = run_both(w, w.T, ctas_per_sm=2)
+    for k in ("gx", "gu", "gv"):
+        assert np.array_equal(a[k], b[k])
+
+
+def test_two_runs_are_bitwise_equal():
+    w = di.mini(di.WORKLOADS["cfg3_adopt_360m"], T=10).replace(K=(2, 3, 4))
+    a = run_both(w, w.T)
+    b = run_both(w, w.T)
+    for k in ("gx", "gu", "gv"):
+        assert np.array_equal(a[k], b[k])
+
+
+@pytest.mark.parametrize("opt", ["adam", "sgdm"])
+@pytest.mark.parametrize("M", [2, 4, 8])
+def test_identical_gradients_match_single_worker_run(opt, M):
+    """Same gradients on every worker: replicas stay bitwise equal to the M = 1 run for any
+    schedule, (1,1,1) "DDP-equivalent" included (fp32 sums of M equal values and the division
+    by M are exact for M a power of two)."""
+    base = di.mini(di.WORKLOADS[f"cfg5_{opt}_ddp"], T=16)
+    for K in [(1, 1, 1), (16, 16, 16), (2, 3, 5)]:
+        many = run_both(base.replace(M=M, K=K), base.T, identical=True)
+        one = run_both(base.replace(M=1, K=K), base.T, identical=True)
+        for k in ("gx", "gu") + (("gv",) if opt != "sgdm" else ()):
+            for m in range(M):
+                assert np.array_equal(many[k][m], one[k][0]), (K, k, m)
+
+
+def test_resume_is_bitwise_identical():
+    """State is the caller's buffers plus the integer t: a fresh context continues a run."""
+    d = _lib()
+    w = di.mini(di.WORKLOADS["cfg2_adam_135m"], T=12).replace(K=(2, 3, 4))
+    full = run_both(w, w.T)
+    dev = torch.device("cuda:0")
+    st = State(w, dev)
+    gv = st.views(st.g)
+    eng = make_engine(d, w, st)
+    for t in range(w.T):
+        if t == w.T // 2:
+            eng.close()
+            eng = make_engine(d, w, st)
+        st.fill_grads(t)
+        eng.step(t, f32r(w.lr), gv)
+    torch.cuda.synchronize()
+    assert np.array_equal(st.to_numpy(st.x), full["gx"])
+    assert np.array_equal(st.to_numpy(st.v), full["gv"])
+    eng.close()
+
+
+# ------------------------------------------------------------------ API behaviour on a device
+def test_gradient_pointers_may_change_every_step_and_lr_schedule():
+    d = _lib()
+    w = di.Workload("swap", "adam", 2, (5000, 33), "bf16", "normal1", lr=1e-2, K=(2, 2, 3), seed=5)
+    dev = torch.device("cuda:0")
+    st = State(w, dev)
+    eng = make_engine(d, w, st)
+    ox, ou, ov = st.to_numpy(st.x), st.to_numpy(st.u), st.to_numpy(st.v)
+    ocfg = oracle_cfg(w)
+    keep = []
+    for t in range(20):                      # more table changes than staging slots
+        st.fill_grads(t)
+        fresh = [b.clone() for b in st.g]    # new addresses every step
+        keep.append(fresh)
+        lr = f32r(1e-2 / (1 + t))
+        eng.step(t, lr, st.views(fresh))
+        oracle.step(ocfg, t, lr, ox, ou, ov, st.to_numpy(fresh))
+    torch.cuda.synchronize()
+    assert rel_err(st.to_numpy(st.x), ox) <= TOL
+    assert rel_err(st.to_numpy(st.v), ov) <= TOL
+    eng.close()
+
+
+def test_errors_are_status_codes_and_context_survives():
+    d = _lib()
+    dev = torch.device("cuda:0")
+    x = torch.zeros(8, device=dev)
+    u = torch.zeros(8, device=dev)
+    v = torch.zeros(8, device=dev)
+    g = torch.ones(8, device=dev)
+    cfg = d.make_config(1, [8], "adam", "f32")
+    ctx = d.desloc_create(cfg, [x.data_ptr()], [u.data_ptr()], [v.data_ptr()], 0)
+    with pytest.raises(d.DeslocError) as e:
+        d.desloc_step(ctx, -1, 1e-3, 0.0, [g.data_ptr()])
+    assert e.value.status == d.DESLOC_E_RANGE
+    with pytest.raises(d.DeslocError) as e:
+        d.desloc_step(ctx, 0, 1e-3, 0.0, [0])
+    assert e.value.status == d.DESLOC_E_NULL
+    with pytest.raises(d.DeslocError) as e:
+        d.desloc_step_masked(ctx, 8, 1e-3, 0.0, [g.data_ptr()])
+    assert e.value.status == d.DESLOC_E_INVALID
+    with pytest.raises(d.DeslocError) as e:
+        d.desloc_step(ctx, 0, float("nan"), 0.0, [g.data_ptr()])
+    assert e.value.status == d.DESLOC_E_RANGE
+    assert d.desloc_step(ctx, 0, 0.5, 0.0, [g.data_ptr()]) == 7
+    torch.cuda.synchronize()
+    assert d.desloc_get_counters(ctx) == [1, 1, 1, 1]
+    # Adam, zero states, g = 1, default eps: u = 0.1, v = 0.001, x = -0.5*0.1/sqrt(0.001)
+    assert torch.allclose(u, torch.full_like(u, 0.1), rtol=1e-6)
+    assert torch.allclose(x, torch.full_like(x, -0.5 * 0.1 / 0.001 ** 0.5), rtol=1e-4)
+    d.desloc_destroy(ctx)
+    d.desloc_destroy(None)
