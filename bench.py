@@ -1,0 +1,433 @@
+#!/usr/bin/env python
+"""DES-LOC step benchmark: G param-updates/s and fraction of the HBM roofline on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One "step" is one call of desloc_step(): the whole hot path (clip, desynced averaging,
+optimizer update for all M worker replicas) over the full synthetic parameter/gradient set.
+Steps run t = 0, 1, 2, ... under the workload's own (K_x, K_u, K_v), so the timed region mixes
+sync and local steps as a run would; per-mask timings (local, x-only, all-sync) are taken
+separately afterwards and reported in "by_mask".
+
+--impl reference times the CPU oracle (the only "reference implementation" this paper has:
+it ships no code) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "desloc_step_param_updates_per_s"
+UNIT = "G param-updates/s"
+NOMINAL_HBM_GBS = 8000.0
+
+
+def bytes_per_param(w) -> int:
+    """Algorithmic HBM bytes per worker-parameter per step: gradient + read and write of each
+    state array (x, u, v fp32; SGDM has no v)."""
+    g = 2 if w.grad_dtype == "bf16" else 4
+    return g + (16 if w.opt == "sgdm" else 24)
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled every 200 ms while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "200", "-i", str(self.idx)], stdout=subprocess.PIPE,
+                stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for ln in self.proc.stdout:
+            self.lines.append((time.time(), ln.strip()))
+
+    def stop(self, t_begin: float, t_end: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        allrows = []
+        for ts, ln in self.lines:
+            f = [a.strip() for a in ln.split(",")]
+            if len(f) < 9:
+                continue
+            allrows.append((ts, f))
+        rows = [r for r in allrows if t_begin <= r[0] <= t_end + 0.2] or allrows
+        for ts, f in rows:
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); pw.append(float(f[3]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "power_w": float(np.median(pw)) if pw else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------ CPU oracle leg
+def time_oracle(w, seconds_target: float = 15.0, threads: int | None = None):
+    """Times the oracle as it stands on this host: `threads` threads, each stepping its own
+    disjoint slice of the workload (same M, optimizer and hyper-parameters, gradients of the
+    workload's distribution), one local step and one all-sync step per round."""
+    import torch
+    import desloc_inputs as di
+    import oracle
+    from concurrent.futures import ThreadPoolExecutor
+    oid = {"adam": oracle.ADAM, "adopt": oracle.ADOPT, "sgdm": oracle.SGDM}[w.opt]
+    threads = threads or max(1, (os.cpu_count() or 1))
+    f32 = lambda a: float(np.float32(a))
+
+    def make_slice(n, seed):
+        ws = w.replace(numel=(n,), seed=seed)
+        x0 = di.init_params(ws).numpy()
+        x = np.ascontiguousarray(np.tile(x0, (w.M, 1)))
+        u = np.zeros_like(x)
+        v = np.zeros_like(x) if w.opt != "sgdm" else None
+        g = torch.empty(w.M, n, dtype=torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32)
+        for m in range(w.M):
+            di.fill_grads_(ws, 0, m, g[m])
+        return x, u, v, np.ascontiguousarray(g.float().numpy())
+
+    def cfg_for(K):
+        return oracle.make_cfg(w.M, oid, beta1=f32(w.beta1), beta2=f32(w.beta2), eps=f32(w.eps),
+                               weight_decay=f32(w.weight_decay), clip_rho=f32(w.clip_rho),
+                               Kx=K[0], Ku=K[1], Kv=K[2],
+                               flags=oracle.FLAG_ADOPT_NORM_CLIP if w.adopt_norm_clip else 0)
+
+    def work(args):
+        x, u, v, g = args
+        # t = 1 with the workload's periods is a local step; t = 0 syncs every array
+        oracle.step(cfg_for(w.K if min(w.K) > 1 else (0, 0, 0)), 1, f32(w.lr), x, u, v, g, clip_bound=1.0)
+        oracle.step(cfg_for(w.K), 0, f32(w.lr), x, u, v, g, clip_bound=1.0)
+
+    # calibrate on a small slice, then size the sample: slices of at most 4 Mi params per
+    # thread (and ~8 GB in total), repeated until ~seconds_target of wall time has passed
+    cal_n = 1 << 15
+    sl = make_slice(cal_n, 1)
+    t0 = time.perf_counter(); work(sl); dt = time.perf_counter() - t0
+    per_elem = dt / (2 * cal_n * w.M)
+    n = int(min(1 << 22, (8 << 30) // (threads * w.M * 16)))
+    n = max(n, 1 << 12)
+    reps = int(max(1, round(seconds_target / (2 * n * w.M * per_elem))))
+    slices = [make_slice(n, 100 + i) for i in range(threads)]
+
+    def work_reps(a):
+        for _ in range(reps):
+            work(a)
+
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        t0 = time.perf_counter()
+        list(ex.map(work_reps, slices))
+        dt = time.perf_counter() - t0
+    updates = 2 * reps * n * w.M * threads
+    return {"value": updates / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"{threads} threads x {n} params x M={w.M} x {2 * reps} steps (alternating "
+                      f"local / all-sync) of {w.name}, {dt:.1f} s", "seconds": dt,
+            "sample_params": n * threads}
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    vals, info = [], None
+    per_step_target = max(2.0, min(20.0, 90.0 / max(1, args.steps + args.warmup)))
+    for i in range(args.warmup + args.steps):
+        info = time_oracle(w, seconds_target=per_step_target)
+        if i >= args.warmup:
+            vals.append(info)
+    value = float(np.mean([v["value"] for v in vals]))
+    # one full-workload step at this rate would take:
+    ms_per_step = w.M * w.N / (value * 1e9) * 1e3
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": w.name, "M": w.M, "params": w.N, "opt": w.opt,
+                   "note": "CPU oracle on host cores; each step is a bounded sample of the "
+                           "workload; ms_per_step extrapolates to the full parameter set"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": info["cores"], "kind": "oracle",
+                         "sample": info["sample"]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ------------------------------------------------------------------------------ GPU leg
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    import desloc_inputs as di
+    import paper_2505_22549_b200 as d
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the DES-LOC step has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- resident state: every rank holds its own M replicas of the whole tensor list -------
+    align = 4
+    nflat = di.flat_size(w.numel, align)
+    offs = di.offsets_of(w.numel, align)
+    gdt = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
+    x0 = di.init_params(w.replace(seed=w.seed + rank), device=dev, align=align)
+    X = [x0.clone() for _ in range(w.M - 1)] + [x0]
+    U = [torch.zeros(nflat, dtype=torch.float32, device=dev) for _ in range(w.M)]
+    V = [torch.zeros(nflat, dtype=torch.float32, device=dev) for _ in range(w.M)] \
+        if w.opt != "sgdm" else None
+    G = [torch.empty(nflat, dtype=gdt, device=dev) for _ in range(w.M)]
+    for m in range(w.M):
+        di.fill_grads_(w.replace(seed=w.seed + rank), 0, m, G[m], align=align)
+    views = lambda bufs: [[b[o:o + n] for o, n in zip(offs, w.numel)] for b in bufs]
+    flags = d.DESLOC_FLAG_ADOPT_NORM_CLIP if w.adopt_norm_clip else 0
+    eng = d.DesLoc(views(X), views(U), views(V) if V is not None else None, opt=w.opt,
+                   grad_dtype=w.grad_dtype, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
+                   weight_decay=w.weight_decay, clip_rho=w.clip_rho, K=w.K, flags=flags)
+    if args.ctas_per_sm is not None:
+        eng.set_launch_shape(args.ctas_per_sm)
+    gv = views(G)
+    bpp = bytes_per_param(w)
+    launch_bytes = w.M * w.N * bpp
+    stream = torch.cuda.current_stream(dev)
+
+    def step(t):
+        return eng.step(t, w.lr, gv, clip_bound=w.clip_bound(t))
+
+    # ---- warm-up: t = 0 (all arrays sync) onwards ---------------------------------------------
+    t_next = 0
+    for _ in range(max(3, args.warmup)):
+        step(t_next); t_next += 1
+    barrier()
+    # the timed window is placed so that one x-sync step falls in its middle, as in a real run
+    Kx = w.K[0]
+    if Kx > 1:
+        t_next = max(t_next, (t_next // Kx + 1) * Kx - args.steps // 2)
+
+    # ---- timed region: exactly K steps, CUDA events on the launching stream -------------------
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    masks = []
+    launches0 = eng.launches()
+    barrier()
+    wall0 = time.time()
+    ev[0].record(stream)
+    for i in range(args.steps):
+        masks.append(step(t_next)); t_next += 1
+        ev[i + 1].record(stream)
+    barrier()
+    wall1 = time.time()
+    launches = eng.launches() - launches0
+    total_ms = ev[0].elapsed_time(ev[-1])
+    per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    clocks = sampler.stop(wall0, wall1) if rank == 0 else None
+    if world > 1:
+        tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+        lt = torch.tensor([launches], dtype=torch.int64, device=dev)
+        dist.all_reduce(lt, op=dist.ReduceOp.SUM)
+        launches = int(lt.item())
+    value = world * w.M * w.N * args.steps / (total_ms * 1e-3) / 1e9
+
+    # ---- per-mask timing (outside the headline region): local, x-only, all-sync ---------------
+    by_mask = {}
+    peak, peak_kind = measured_peak()
+    masks_to_time = [0, 1, 3 if w.opt == "sgdm" else 7]
+    reps = max(3, min(args.steps, 10))
+    for mk in masks_to_time:
+        if w.M == 1 and mk:
+            continue
+        for _ in range(2):
+            eng.step_masked(mk, w.lr, gv, clip_bound=1.0)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            eng.step_masked(mk, w.lr, gv, clip_bound=1.0)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        gbs = launch_bytes / (ms * 1e-3) / 1e9
+        by_mask[str(mk)] = {"ms": ms, "gups": w.M * w.N / (ms * 1e-3) / 1e9, "gbs": gbs,
+                            "frac_of_measured_peak": gbs / peak,
+                            "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS}
+
+    # ---- roofline of the dominant kernel (the local-step kernel), from the timed region -------
+    local_ms = [ms for ms, mk in zip(per_step, masks) if mk == 0] or per_step
+    avg_local_ms = float(np.mean(local_ms))
+    achieved = launch_bytes / (avg_local_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": TRAFFIC_BYTES.get(w.name),
+                "peak_source": f"{peak_kind} copy bandwidth", "kernel": "desloc_step_kernel (local step)",
+                "algorithmic_bytes_per_launch": launch_bytes,
+                "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
+                "avg_launch_ms": avg_local_ms, "launches_averaged": len(local_ms)}
+
+    # ---- end to end: gradients start in pinned host memory, a result is read back -------------
+    e2e = run_e2e(args, w, eng, G, X, offs, dev, world, barrier)
+
+    if rank == 0:
+        cpu = time_oracle(w, seconds_target=15.0)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": w.name, "opt": w.opt, "M": w.M, "params": w.N,
+                       "tensors": len(w.numel), "grad_dtype": w.grad_dtype, "K": list(w.K),
+                       "resident_gb": w.M * w.N * (bpp - (8 if w.opt == "sgdm" else 12)) / 1e9,
+                       "l2": "inputs larger than L2 (no flush needed)",
+                       "parallelism": f"{world} independent replica set(s), no collective",
+                       "masks_in_timed_region": masks},
+            "roofline": roofline, "by_mask": by_mask, "cpu_baseline": {k: cpu[k] for k in
+                                                                       ("value", "unit", "cores", "kind", "sample")},
+            "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+        }
+        print(json.dumps(line), flush=True)
+    eng.close()
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+# DRAM bytes (read + write) of one launch of the local-step kernel, from an ncu capture
+# summarised under profiles/; filled in per workload once measured.
+TRAFFIC_BYTES: dict = {}
+
+
+def run_e2e(args, w, eng, G, X, offs, dev, world, barrier):
+    """Same step, but every step's gradients are copied from pinned host memory first and a
+    small result (worker 0's last tensor of x) is read back to the host afterwards."""
+    import torch
+    esz = G[0].element_size()
+    nflat = G[0].numel()
+    h2d = w.M * nflat * esz
+    try:
+        import psutil
+        avail = psutil.virtual_memory().available
+    except Exception:
+        avail = 0
+    share = h2d + (8 << 30) < avail / max(1, world)
+    try:
+        if share:
+            H = [torch.empty(nflat, dtype=G[0].dtype).pin_memory() for _ in range(w.M)]
+        else:
+            H = [torch.empty(nflat, dtype=G[0].dtype).pin_memory()] * w.M
+        for h, g in zip(H[:w.M if share else 1], G):
+            h.copy_(g)
+    except Exception as ex:  # not enough pinnable memory on this host
+        return {"value": None, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 0,
+                "note": f"pinned host buffer unavailable: {type(ex).__name__}"}
+    stream = torch.cuda.current_stream(dev)
+    views = lambda bufs: [[b[o:o + n] for o, n in zip(offs, w.numel)] for b in bufs]
+    gv = views(G)
+    last = (offs[-1], w.numel[-1])
+    out = torch.empty(last[1], dtype=torch.float32).pin_memory()
+    steps = max(2, min(args.steps, 6))
+    t_next = 1000
+
+    def one(t):
+        for m in range(w.M):
+            G[m].copy_(H[m], non_blocking=True)
+        eng.step(t, w.lr, gv, clip_bound=w.clip_bound(t))
+        out.copy_(X[0][last[0]:last[0] + last[1]], non_blocking=True)
+        stream.synchronize()
+
+    one(t_next); t_next += 1
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        one(t_next); t_next += 1
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    if world > 1:
+        import torch.distributed as dist
+        tt = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms = float(tt.item())
+    return {"value": world * w.M * w.N * steps / (ms * 1e-3) / 1e9, "unit": UNIT,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": last[1] * 4, "steps": steps,
+            "ms_per_step": ms / steps,
+            "note": "gradients copied from pinned host memory every step"
+                    + ("" if share else " (one host buffer re-sent for each worker)")}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4_adam_1p7b")
+    ap.add_argument("--ctas-per-sm", type=int, default=None)
+    args = ap.parse_args()
+    import desloc_inputs as di
+    w = di.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        return run_reference(args, w)
+    return run_ours(args, w)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

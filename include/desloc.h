@@ -9,8 +9,8 @@
  * This library keeps all M worker replicas in ONE GPU's memory.  One call to
  * desloc_step() runs one step t of Algorithm 1 for all workers: a single
  * memory-bound kernel reads g, x, u, v of every replica once, clips the
- * gradient, averages the arrays whose period divides t in registers (fixed
- * order m = 0..M-1), applies the per-worker update and writes x, u, v back.
+ * gradient, averages the arrays whose period divides t in registers (a fixed
+ * summation tree over m), applies the per-worker update and writes x, u, v back.
  * A sync step therefore moves the same bytes as a local step; there is no
  * separate averaging pass and no collective.
  *

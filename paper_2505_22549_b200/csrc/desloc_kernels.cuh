@@ -6,7 +6,7 @@
 //   * local steps (no array synced) treat workers independently: the work item is
 //     (worker, chunk) and the kernel is the MT = 1 instantiation;
 //   * sync steps are instantiated per worker count MT = M and per sync mask: a thread loads
-//     its elements of all M replicas, sums the synced arrays in the fixed order m = 0..M-1,
+//     its elements of all M replicas, sums the synced arrays in a fixed tree order,
 //     and writes every replica back -- the same bytes as a local step.
 // Every thread issues all loads of its tile (MT workers x UN positions x 4 arrays, 128-bit
 // where aligned) before the first use, so that enough bytes are in flight to cover HBM
@@ -103,13 +103,24 @@ __device__ __forceinline__ FV<VEC> ld_grad(const char *base, long long elem) {
 // ---- the update of one coordinate across all MT workers (registers only) -----------------
 // Pre-average (Algorithms 1-3): synced arrays are replaced by their worker mean BEFORE the
 // update.  Post-average (Algorithms 4-5): the updated values are averaged, and the parameter
-// step uses the averaged states.  Sums run m = 0..MT-1 in that order.
+// step uses the averaged states.
+// Worker sum as a fixed binary tree: the first 2^k workers (2^k the largest power of two
+// below the count) against the rest, recursively -- ((s0+s1)+(s2+s3))+((s4+s5)+(s6+s7)) for
+// eight.  Deterministic, and exact when all M values are equal and M is a power of two.
+template <int LO, int N, int MT>
+__device__ __forceinline__ float tree_sum(const float (&s)[MT]) {
+    if constexpr (N == 1) {
+        return s[LO];
+    } else {
+        constexpr int H = (N > 4) ? 4 : (N > 2 ? 2 : 1);
+        static_assert(N <= 8, "tree_sum covers up to eight workers");
+        return tree_sum<LO, H, MT>(s) + tree_sum<LO + H, N - H, MT>(s);
+    }
+}
+
 template <int MT>
 __device__ __forceinline__ float mean_of(const float (&s)[MT]) {
-    float acc = s[0];
-#pragma unroll
-    for (int m = 1; m < MT; ++m) acc += s[m];
-    return acc / static_cast<float>(MT);
+    return tree_sum<0, MT, MT>(s) / static_cast<float>(MT);
 }
 
 template <int OPT, int MASK, int MT, bool POST>
