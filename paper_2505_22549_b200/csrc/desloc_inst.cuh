@@ -13,20 +13,24 @@ const void *kernel_ptr() {
     return reinterpret_cast<const void *>(&desloc_step_kernel<OPT, MASK, MT, GT, POST>);
 }
 
-// NMASK = 7 (masks 1..7) for Adam / ADOPT, 3 (masks 1..3: no second state) for SGDM.
-template <int OPT, bool POST, typename GT, int NMASK, int... I>
+// Masks FIRST..LAST for every MT in 2..MAX_MT.  LAST = 7 for Adam / ADOPT, 3 for SGDM (no
+// second state).  FIRST = 0 for the pre-average units (mask 0, the local step, is the same
+// code for either ordering) and 1 for the post-average ones.
+template <int OPT, bool POST, typename GT, int FIRST, int NMASK, int... I>
 const void *pick_sync(int mt, int mask, std::integer_sequence<int, I...>) {
-    static const void *const tbl[] = {kernel_ptr<OPT, POST, GT, 2 + I / NMASK, 1 + I % NMASK>()...};
-    if (mt < 2 || mt > MAX_MT || mask < 1 || mask > NMASK) return nullptr;
-    return tbl[(mt - 2) * NMASK + (mask - 1)];
+    static const void *const tbl[] = {
+        kernel_ptr<OPT, POST, GT, 2 + I / NMASK, FIRST + I % NMASK>()...};
+    if (mt < 2 || mt > MAX_MT || mask < FIRST || mask >= FIRST + NMASK) return nullptr;
+    return tbl[(mt - 2) * NMASK + (mask - FIRST)];
 }
 
 template <int OPT, bool POST>
 const void *lookup_sync(bool bf16, int mt, int mask) {
-    constexpr int NMASK = (OPT == OPT_SGDM) ? 3 : 7;
+    constexpr int FIRST = POST ? 1 : 0;
+    constexpr int NMASK = ((OPT == OPT_SGDM) ? 3 : 7) + 1 - FIRST;
     using Seq = std::make_integer_sequence<int, (MAX_MT - 1) * NMASK>;
-    return bf16 ? pick_sync<OPT, POST, bf16_t, NMASK>(mt, mask, Seq{})
-                : pick_sync<OPT, POST, float, NMASK>(mt, mask, Seq{});
+    return bf16 ? pick_sync<OPT, POST, bf16_t, FIRST, NMASK>(mt, mask, Seq{})
+                : pick_sync<OPT, POST, float, FIRST, NMASK>(mt, mask, Seq{});
 }
 
 template <int OPT>

@@ -3,11 +3,12 @@
 //
 // Work decomposition.  The tensor list is cut into chunks of CHUNK_ELEMS elements of one
 // tensor (table built once on the host).  A thread block takes one chunk at a time:
-//   * local steps (no array synced) treat workers independently: the work item is
-//     (worker, chunk) and the kernel is the MT = 1 instantiation;
-//   * sync steps are instantiated per worker count MT = M and per sync mask: a thread loads
-//     its elements of all M replicas, sums the synced arrays in a fixed tree order,
-//     and writes every replica back -- the same bytes as a local step.
+//   * for M = 2..8 the kernel is instantiated per worker count MT = M and per sync mask
+//     (mask 0 = local step): a thread loads its elements of all M replicas, sums the synced
+//     arrays in a fixed tree order, and writes every replica back -- a sync step moves the
+//     same bytes as a local step, through the same code shape;
+//   * the MT = 1 instantiation serves M = 1 and local steps of M > 8: workers are
+//     independent there, so the work item is (worker, chunk).
 // Every thread issues all loads of its tile (MT workers x UN positions x 4 arrays, 128-bit
 // where aligned) before the first use, so that enough bytes are in flight to cover HBM
 // latency; the arithmetic is fp32.  Tensors whose pointers are not 16-byte aligned and the
@@ -302,8 +303,7 @@ desloc_step_kernel(const __grid_constant__ StepArgs a) {
 }
 
 // Lookup of an instantiation: opt, post-average?, bf16 gradients?, MT in 1..MAX_MT, mask.
-// MT == 1 exists only with mask 0 (the mean of one replica is itself).  Returns nullptr for
-// combinations that do not exist.
+// Returns nullptr for combinations that do not exist (sync masks with M > MAX_MT).
 const void *lookup_step_kernel(int opt, bool post, bool bf16, int mt, int mask);
 
 }  // namespace desloc
