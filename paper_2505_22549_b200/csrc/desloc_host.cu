@@ -18,10 +18,13 @@ namespace desloc {
 
 const void *lookup_step_kernel(int opt, bool post, bool bf16, int mt, int mask) {
     if (mask == 0) {
-        // Local step: the same code for either ordering and any M.
-        if (opt == OPT_ADAM) return lookup_adam_pre(bf16, 1, 0);
-        if (opt == OPT_ADOPT) return lookup_adopt_pre(bf16, 1, 0);
-        if (opt == OPT_SGDM) return lookup_sgdm_pre(bf16, 1, 0);
+        // Local step: the same code for either ordering.  Up to MAX_MT workers it uses the
+        // all-workers-per-chunk instantiation (more bytes per block and per pointer set-up);
+        // beyond that, and for M = 1, workers are separate work items of the MT = 1 kernel.
+        const int m = (mt >= 2 && mt <= MAX_MT) ? mt : 1;
+        if (opt == OPT_ADAM) return lookup_adam_pre(bf16, m, 0);
+        if (opt == OPT_ADOPT) return lookup_adopt_pre(bf16, m, 0);
+        if (opt == OPT_SGDM) return lookup_sgdm_pre(bf16, m, 0);
         return nullptr;
     }
     if (opt == OPT_ADAM) return post ? lookup_adam_post(bf16, mt, mask) : lookup_adam_pre(bf16, mt, mask);
@@ -169,8 +172,9 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
         // The mean of one replica is the replica: M = 1 always runs the local kernel.
         const uint32_t kmask = (c.M == 1) ? 0u : mask;
         const bool post = (c.flags & DESLOC_FLAG_POST_AVERAGE) != 0;
+        const bool per_worker_items = (c.M == 1) || (kmask == 0 && c.M > desloc::MAX_MT);
         const void *fn = desloc::lookup_step_kernel(c.opt, post, c.grad_dtype == DESLOC_BF16,
-                                                    kmask ? c.M : 1, static_cast<int>(kmask));
+                                                    c.M, static_cast<int>(kmask));
         if (!fn) {
             rc = DESLOC_E_INVALID;
             break;
@@ -195,7 +199,7 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
         a.rho = c.clip_rho > 0.f ? c.clip_rho : std::numeric_limits<float>::infinity();
         a.cbound = nclip ? clip_bound_t : std::numeric_limits<float>::infinity();
 
-        const long long nitems = kmask ? ctx->nchunks : ctx->nchunks * c.M;
+        const long long nitems = per_worker_items ? ctx->nchunks * c.M : ctx->nchunks;
         long long grid = nitems;
         if (ctx->ctas_per_sm > 0) {
             const long long cap = static_cast<long long>(ctx->ctas_per_sm) * ctx->num_sms;
