@@ -72,7 +72,8 @@ typedef enum {
     DESLOC_E_RANGE = -2,   /* M, a period, a beta, eps, weight decay, numel or t out of range */
     DESLOC_E_INVALID = -3, /* unknown optimizer / dtype / flag, or a flag the optimizer lacks */
     DESLOC_E_NOMEM = -4,   /* host or device allocation failed */
-    DESLOC_E_CUDA = -5     /* a CUDA call failed; see desloc_last_cuda_error() */
+    DESLOC_E_CUDA = -5,    /* a CUDA call failed; see desloc_last_cuda_error() */
+    DESLOC_E_TOO_LARGE = -6 /* desloc_step_static(): the problem exceeds the fixed scratch */
 } desloc_status;
 
 /* The "Require" block of Algorithms 1-3: everything fixed for a run.  Plain data, copied
@@ -167,6 +168,46 @@ DESLOC_API int64_t desloc_plan_chunks(const int64_t *numel, int32_t num_tensors,
 
 /* Elements per chunk used by contexts of this build. */
 DESLOC_API int64_t desloc_chunk_elems(void);
+
+/*
+ * desloc_step_static(): one step for callers that cannot allocate.  (The paper has no
+ * counterpart; this is an interface variant, the update computed is desloc_step()'s.)
+ *
+ * desloc_create() takes device memory for its chunk and pointer tables.  That is not possible
+ * for every caller: a process whose training framework has already claimed all of HBM for its
+ * own memory pool gets an out-of-memory error from any further cudaMalloc (or forces the pool
+ * to give memory back), and a latency-critical loop cannot afford the device-wide
+ * synchronisation that cudaMalloc and cudaFree bring.  This entry point needs no context and
+ * calls no cudaMalloc, cudaFree, cudaMallocHost or any other allocating routine: its tables
+ * go into a fixed array inside the library image, DESLOC_STATIC_SCRATCH_BYTES (about 320 KB)
+ * of device memory that every GPU which loads the library holds until the process exits.
+ *
+ * Limits: M * num_tensors <= DESLOC_STATIC_MAX_POINTERS, M <= 8, and at most
+ * DESLOC_STATIC_MAX_CHUNKS chunks of desloc_chunk_elems() elements (every tensor starts a new
+ * chunk) -- up to 64 Mi parameters when tensors are large.  Anything bigger returns
+ * DESLOC_E_TOO_LARGE and does nothing.
+ *
+ * Arguments as for desloc_create() + desloc_step(): cfg, the host arrays x, u, v, grads of
+ * M*num_tensors DEVICE pointers (v may be NULL for SGDM), the step t, eta_t, the ADOPT bound,
+ * the device and the stream.  State is updated in place; nothing is remembered between calls,
+ * so there are no counters.  The tables are built on the calling thread's stack (about 320 KB
+ * of it) and copied to the device on `stream` ahead of the kernel.
+ *
+ * The first call on each device looks up the device address of the scratch array
+ * (cudaGetSymbolAddress, with that device current); make that first call before any stream
+ * capture begins.  All calls on a device share the one array and it keeps the previous
+ * call's tables: each call rewrites the part it uses, nothing in it needs to start at zero.
+ * Two calls whose GPU work can overlap -- different streams without an ordering between them,
+ * or two host threads -- race on the array and must be serialised by the caller; calls issued
+ * one after the other on the same stream are safe.
+ */
+#define DESLOC_STATIC_MAX_POINTERS 2048
+#define DESLOC_STATIC_MAX_CHUNKS 16384
+#define DESLOC_STATIC_SCRATCH_BYTES (DESLOC_STATIC_MAX_CHUNKS * 16 + 4 * DESLOC_STATIC_MAX_POINTERS * 8)
+DESLOC_API int desloc_step_static(const desloc_config *cfg, float *const *x, float *const *u,
+                                  float *const *v, const void *const *grads, int64_t t,
+                                  float lr_t, float clip_bound_t, int cuda_device, void *stream,
+                                  uint32_t *mask_out);
 
 /* Static description of a status code; never NULL. */
 DESLOC_API const char *desloc_strerror(int status);

@@ -20,6 +20,8 @@ DESLOC_SYNC_X, DESLOC_SYNC_U, DESLOC_SYNC_V = 1, 2, 4
 DESLOC_FLAG_ADOPT_NORM_CLIP, DESLOC_FLAG_POST_AVERAGE = 1, 2
 DESLOC_OK, DESLOC_E_NULL, DESLOC_E_RANGE, DESLOC_E_INVALID, DESLOC_E_NOMEM, DESLOC_E_CUDA = \
     0, -1, -2, -3, -4, -5
+DESLOC_E_TOO_LARGE = -6
+DESLOC_STATIC_MAX_POINTERS, DESLOC_STATIC_MAX_CHUNKS = 2048, 16384
 DESLOC_MAX_M = 64
 
 OPT_BY_NAME = {"adam": DESLOC_ADAM, "adopt": DESLOC_ADOPT, "sgdm": DESLOC_SGDM}
@@ -75,6 +77,10 @@ _lib.desloc_step_masked.restype = ctypes.c_int
 _lib.desloc_step_masked.argtypes = [_P, ctypes.c_uint32, ctypes.c_float, ctypes.c_float, _PP, _P]
 _lib.desloc_destroy.restype = ctypes.c_int
 _lib.desloc_destroy.argtypes = [_P]
+_lib.desloc_step_static.restype = ctypes.c_int
+_lib.desloc_step_static.argtypes = [ctypes.POINTER(DeslocConfig), _PP, _PP, _PP, _PP,
+                                    ctypes.c_int64, ctypes.c_float, ctypes.c_float, ctypes.c_int,
+                                    _P, ctypes.POINTER(ctypes.c_uint32)]
 _lib.desloc_get_counters.restype = ctypes.c_int
 _lib.desloc_get_counters.argtypes = [_P, ctypes.POINTER(ctypes.c_int64)]
 _lib.desloc_get_launch_count.restype = ctypes.c_int64
@@ -155,6 +161,23 @@ def desloc_step_masked(ctx: int, mask: int, lr_t: float, clip_bound_t: float, gr
                                  stream or None)
     if rc != DESLOC_OK:
         raise DeslocError(rc, "desloc_step_masked", _lib.desloc_last_cuda_error(ctx))
+
+
+def desloc_step_static(cfg: DeslocConfig, x, u, v, grads, t: int, lr_t: float,
+                       clip_bound_t: float, cuda_device: int, stream: int = 0) -> int:
+    """One step with no context and no allocation (tables go to the library's fixed device
+    array).  x, u, v, grads: sequences of device pointers, entry m*num_tensors + k.  Returns
+    the sync mask; raises DeslocError (DESLOC_E_TOO_LARGE beyond the fixed capacity).  Calls
+    that may overlap on the GPU must be serialised by the caller."""
+    mask = ctypes.c_uint32(0)
+    as_arr = lambda a: a if isinstance(a, ctypes.Array) else _ptr_array(a)
+    rc = _lib.desloc_step_static(ctypes.byref(cfg) if cfg is not None else None, as_arr(x),
+                                 as_arr(u), as_arr(v), as_arr(grads), int(t), float(lr_t),
+                                 float(clip_bound_t), int(cuda_device), stream or None,
+                                 ctypes.byref(mask))
+    if rc != DESLOC_OK:
+        raise DeslocError(rc, "desloc_step_static")
+    return int(mask.value)
 
 
 def desloc_destroy(ctx: Optional[int]) -> None:

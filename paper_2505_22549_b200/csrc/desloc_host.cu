@@ -399,6 +399,7 @@ const char *desloc_strerror(int status) {
         case DESLOC_E_INVALID: return "invalid optimizer, dtype, flag or mask";
         case DESLOC_E_NOMEM: return "out of memory";
         case DESLOC_E_CUDA: return "CUDA call failed";
+        case DESLOC_E_TOO_LARGE: return "problem exceeds the fixed scratch of desloc_step_static";
         default: return "unknown status";
     }
 }
