@@ -98,6 +98,14 @@ def _wl() -> dict:
         for tag, K in (("ddp", (1, 1, 1)), ("local", (16, 16, 16)), ("desloc", (16, 64, 256))):
             name = f"cfg5_{opt}_{tag}"
             w[name] = base5.replace(name=name, opt=opt, K=K)
+    # Small stand-ins of workloads 4 and 3 for profiler captures: same optimizer, M, dtypes and
+    # gradient recipe on a 6-block model (44 M parameters; 2.5 / 4.9 GB resident, well above
+    # the 126 MB L2, small enough for a multi-pass capture).
+    prof = tuple(llama_tensor_list(6, 768, 256, 2048, 8192))
+    w["prof_adam_m4_44m"] = w["cfg4_adam_1p7b"].replace(name="prof_adam_m4_44m", numel=prof,
+                                                        K=(4, 8, 16), T=16)
+    w["prof_adopt_m8_44m"] = w["cfg3_adopt_360m"].replace(name="prof_adopt_m8_44m", numel=prof,
+                                                          K=(4, 8, 16), T=16)
     return w
 
 
