@@ -173,8 +173,11 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
         const uint32_t kmask = (c.M == 1) ? 0u : mask;
         const bool post = (c.flags & DESLOC_FLAG_POST_AVERAGE) != 0;
         const bool per_worker_items = (c.M == 1) || (kmask == 0 && c.M > desloc::MAX_MT);
-        const void *fn = desloc::lookup_step_kernel(c.opt, post, c.grad_dtype == DESLOC_BF16,
-                                                    c.M, static_cast<int>(kmask));
+        const bool generic = kmask != 0 && c.M > desloc::MAX_MT;
+        const void *fn = generic
+                             ? desloc::lookup_generic_kernel(c.opt, post, c.grad_dtype == DESLOC_BF16)
+                             : desloc::lookup_step_kernel(c.opt, post, c.grad_dtype == DESLOC_BF16,
+                                                          c.M, static_cast<int>(kmask));
         if (!fn) {
             rc = DESLOC_E_INVALID;
             break;
@@ -206,7 +209,8 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
             if (grid > cap) grid = cap;
         }
         if (grid > 0x7fffffffLL) grid = 0x7fffffffLL;  // the kernel strides over the rest
-        void *params[] = {&a};
+        int kmask_arg = static_cast<int>(kmask);
+        void *params[] = {&a, &kmask_arg};  // the second one is read by the generic kernel only
         e = cudaLaunchKernel(fn, dim3(static_cast<unsigned>(grid)), dim3(desloc::BLOCK_THREADS),
                              params, 0, stream);
         if (e != cudaSuccess) {

@@ -306,4 +306,7 @@ desloc_step_kernel(const __grid_constant__ StepArgs a) {
 // Returns nullptr for combinations that do not exist (sync masks with M > MAX_MT).
 const void *lookup_step_kernel(int opt, bool post, bool bf16, int mt, int mask);
 
+// Runtime-M kernel for sync steps of M > MAX_MT; launched with (StepArgs, int mask).
+const void *lookup_generic_kernel(int opt, bool post, bool bf16);
+
 }  // namespace desloc

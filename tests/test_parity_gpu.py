@@ -128,6 +128,31 @@ def test_post_average_ordering(opt, M):
             assert np.array_equal(res[a][0], res[a][m])
 
 
+@pytest.mark.parametrize("opt", ["adam", "adopt", "sgdm"])
+@pytest.mark.parametrize("M,post", [(9, False), (16, False), (16, True), (33, True), (64, False)])
+def test_many_workers_runtime_m_path(opt, M, post):
+    """More workers than the register-resident kernels hold (M > 8): runtime-M kernel on sync
+    steps, per-worker items on local steps; up to the largest M a context accepts."""
+    numel = (3, 4096, 4101, 777)
+    nmask = 4 if opt == "sgdm" else 8
+    masks = list(range(nmask)) + [nmask - 1, 0]
+    w = di.Workload(f"many_{opt}", opt, M, numel, "bf16", "normal1", beta1=0.9, beta2=0.99,
+                    eps=1e-2, lr=1e-2, weight_decay=0.01, clip_rho=2.0,
+                    adopt_norm_clip=(opt == "adopt"), seed=11 + M)
+    for align in (4, 1):
+        res = run_both(w, len(masks), align=align, forced_masks=masks, post=post, v_init=0.5)
+        check(res)
+
+
+def test_identical_gradients_with_sixteen_workers_match_single_worker():
+    base = di.mini(di.WORKLOADS["cfg5_adam_ddp"], T=8).replace(K=(1, 2, 3))
+    many = run_both(base.replace(M=16), base.T, identical=True)
+    one = run_both(base.replace(M=1), base.T, identical=True)
+    for k in ("gx", "gu", "gv"):
+        for m in range(16):
+            assert np.array_equal(many[k][m], one[k][0])
+
+
 def test_misaligned_buffers_take_the_scalar_path():
     w = di.Workload("shift", "adam", 3, (4096 * 2 + 5, 17), "bf16", "normal1", lr=1e-2,
                     K=(2, 3, 4), seed=3)
