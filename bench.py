@@ -428,11 +428,15 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4_adam_1p7b")
     ap.add_argument("--ctas-per-sm", type=int, default=None)
+    ap.add_argument("--workers", type=int, default=None,
+                    help="override the workload's worker count M (exploration only)")
     ap.add_argument("--skip-e2e", action="store_true", help="omit the host-buffer leg (profiling)")
     ap.add_argument("--skip-cpu", action="store_true", help="omit the CPU oracle leg (profiling)")
     args = ap.parse_args()
     import desloc_inputs as di
     w = di.WORKLOADS[args.workload]
+    if args.workers:
+        w = w.replace(name=f"{w.name}_M{args.workers}", M=args.workers)
     if args.impl == "reference":
         return run_reference(args, w)
     return run_ours(args, w)

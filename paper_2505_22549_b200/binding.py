@@ -12,7 +12,8 @@ import os
 from typing import Optional, Sequence
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "lib", "libdesloc.so")
+# DESLOC_LIBRARY selects another build of the same library (e.g. a tuning variant).
+LIB_PATH = os.environ.get("DESLOC_LIBRARY") or os.path.join(_HERE, "lib", "libdesloc.so")
 
 DESLOC_ADAM, DESLOC_ADOPT, DESLOC_SGDM = 0, 1, 2
 DESLOC_F32, DESLOC_BF16 = 0, 1

@@ -49,16 +49,34 @@ def _fingerprint(src: str) -> str:
     return h.hexdigest()
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, extra_flags=(), out: str | None = None,
+          obj_dir: str | None = None) -> str:
+    """Compile every translation unit (in parallel) and link the shared library.
+
+    extra_flags / out / obj_dir build a tuning variant (e.g. -DDESLOC_MINB_LARGE_M=3) into
+    another file without touching the default library."""
+    global OBJ, LIB
+    saved = (OBJ, LIB)
+    if obj_dir:
+        OBJ = obj_dir
+    if out:
+        LIB = out
+    try:
+        return _build(force, verbose, list(extra_flags))
+    finally:
+        OBJ, LIB = saved
+
+
+def _build(force: bool, verbose: bool, extra_flags) -> str:
     os.makedirs(OBJ, exist_ok=True)
-    os.makedirs(LIBDIR, exist_ok=True)
+    os.makedirs(os.path.dirname(LIB), exist_ok=True)
     nvcc = _nvcc()
-    flags = NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else [])
+    flags = NVCC_FLAGS + extra_flags + (["-Xptxas", "-v"] if verbose else [])
 
     def compile_one(src):
         obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
         stamp = obj + ".stamp"
-        fp = _fingerprint(src)
+        fp = _fingerprint(src) + " ".join(extra_flags)
         if (not force and os.path.exists(obj) and os.path.exists(stamp)
                 and open(stamp).read() == fp):
             return obj, False

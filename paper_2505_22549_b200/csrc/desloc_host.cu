@@ -202,7 +202,9 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
         a.rho = c.clip_rho > 0.f ? c.clip_rho : std::numeric_limits<float>::infinity();
         a.cbound = nclip ? clip_bound_t : std::numeric_limits<float>::infinity();
 
-        const long long nitems = per_worker_items ? ctx->nchunks * c.M : ctx->nchunks;
+        const long long nitems =
+            per_worker_items ? ((ctx->nchunks + desloc::LOCAL_SLOTS - 1) / desloc::LOCAL_SLOTS) * c.M
+                             : ctx->nchunks;
         long long grid = nitems;
         if (ctx->ctas_per_sm > 0) {
             const long long cap = static_cast<long long>(ctx->ctas_per_sm) * ctx->num_sms;

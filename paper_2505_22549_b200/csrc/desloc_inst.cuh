@@ -35,7 +35,8 @@ const void *lookup_sync(bool bf16, int mt, int mask) {
 
 template <int OPT>
 const void *lookup_local(bool bf16) {
-    return bf16 ? kernel_ptr<OPT, false, bf16_t, 1, 0>() : kernel_ptr<OPT, false, float, 1, 0>();
+    return bf16 ? reinterpret_cast<const void *>(&desloc_local_kernel<OPT, bf16_t>)
+                : reinterpret_cast<const void *>(&desloc_local_kernel<OPT, float>);
 }
 
 const void *lookup_adam_pre(bool bf16, int mt, int mask);

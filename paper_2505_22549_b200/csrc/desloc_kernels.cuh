@@ -7,8 +7,8 @@
 //     (mask 0 = local step): a thread loads its elements of all M replicas, sums the synced
 //     arrays in a fixed tree order, and writes every replica back -- a sync step moves the
 //     same bytes as a local step, through the same code shape;
-//   * the MT = 1 instantiation serves M = 1 and local steps of M > 8: workers are
-//     independent there, so the work item is (worker, chunk).
+//   * desloc_local_kernel serves M = 1 and local steps of M > 8: workers are independent
+//     there, so the work item is (worker, group of four consecutive chunks).
 // Every thread issues all loads of its tile (MT workers x UN positions x 4 arrays, 128-bit
 // where aligned) before the first use, so that enough bytes are in flight to cover HBM
 // latency; the arithmetic is fp32.  Tensors whose pointers are not 16-byte aligned and the
@@ -16,6 +16,17 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+
+// Tuning of the MT > 4 instantiations (measured on B200, 360 M parameters x 8 workers): Adam
+// and ADOPT run the batched tile below at three blocks per SM (97 % of copy bandwidth against
+// 94-95 % for the all-at-once tile, which spills at 128 registers); SGDM, with one state less,
+// is fastest all-at-once at two blocks per SM (98 %).
+#ifndef DESLOC_SPLIT_LARGE_M
+#define DESLOC_SPLIT_LARGE_M 1
+#endif
+#ifndef DESLOC_MINB_LARGE_M
+#define DESLOC_MINB_LARGE_M 3
+#endif
 
 namespace desloc {
 
@@ -124,6 +135,40 @@ __device__ __forceinline__ float mean_of(const float (&s)[MT]) {
     return tree_sum<0, MT, MT>(s) / static_cast<float>(MT);
 }
 
+// One worker's state update from the clipped gradient: `up`, `vp` are the previous states the
+// update starts from (the worker's own or the worker mean); `vown` is always the worker's own
+// previous v, which ADOPT's normaliser uses (Algorithm 3).
+template <int OPT>
+__device__ __forceinline__ void state_update(const StepArgs &a, float g, float up, float vp,
+                                             float vown, float &un, float &vn) {
+    // coordinate-wise clip: sgn(g) min(|g|, rho)  (Section 3.1); rho = +inf when off
+    const float gh = fminf(fmaxf(g, -a.rho), a.rho);
+    if constexpr (OPT == OPT_ADAM) {
+        un = fmaf(a.b1, up, a.omb1 * gh);
+        vn = fmaf(a.b2, vp, (a.omb2 * gh) * gh);
+    } else if constexpr (OPT == OPT_ADOPT) {
+        vn = fmaf(a.b2, vp, (a.omb2 * gh) * gh);
+        float r = gh / fmaxf(sqrtf(vown), a.eps);
+        r = fminf(fmaxf(r, -a.cbound), a.cbound);
+        un = fmaf(a.b1, up, a.omb1 * r);
+    } else {
+        un = fmaf(a.b1, up, a.omb1 * gh);
+        vn = 0.f;
+    }
+}
+
+// One worker's parameter step from base xp with the new states.
+template <int OPT>
+__device__ __forceinline__ float param_step(const StepArgs &a, float xp, float un, float vn) {
+    float d;
+    if constexpr (OPT == OPT_ADAM)
+        d = (a.lr * un) / sqrtf(vn + a.lam2);
+    else
+        d = a.lr * un;
+    // x* (1 - eta wd) - d, written as x* - (eta wd x* + d): one rounding at x's scale
+    return xp - fmaf(a.lrwd, xp, d);
+}
+
 template <int OPT, int MASK, int MT, bool POST>
 __device__ __forceinline__ void update_coord(const StepArgs &a, const float (&g)[MT],
                                              float (&x)[MT], float (&u)[MT], float (&v)[MT]) {
@@ -136,24 +181,9 @@ __device__ __forceinline__ void update_coord(const StepArgs &a, const float (&g)
     float un[MT], vn[MT], xn[MT];
 #pragma unroll
     for (int m = 0; m < MT; ++m) {
-        // coordinate-wise clip: sgn(g) min(|g|, rho)  (Section 3.1); rho = +inf when off
-        const float gh = fminf(fmaxf(g[m], -a.rho), a.rho);
         const float up = (PRE && (MASK & SYNC_U)) ? ub : u[m];
-        if constexpr (OPT == OPT_ADAM) {
-            const float vp = (PRE && (MASK & SYNC_V)) ? vb : v[m];
-            un[m] = fmaf(a.b1, up, a.omb1 * gh);
-            vn[m] = fmaf(a.b2, vp, (a.omb2 * gh) * gh);
-        } else if constexpr (OPT == OPT_ADOPT) {
-            const float vp = (PRE && (MASK & SYNC_V)) ? vb : v[m];
-            vn[m] = fmaf(a.b2, vp, (a.omb2 * gh) * gh);
-            // normalised by the worker's own v from before this step
-            float r = gh / fmaxf(sqrtf(v[m]), a.eps);
-            r = fminf(fmaxf(r, -a.cbound), a.cbound);
-            un[m] = fmaf(a.b1, up, a.omb1 * r);
-        } else {
-            un[m] = fmaf(a.b1, up, a.omb1 * gh);
-            vn[m] = 0.f;
-        }
+        const float vp = (PRE && (MASK & SYNC_V)) ? vb : v[m];
+        state_update<OPT>(a, g[m], up, vp, v[m], un[m], vn[m]);
     }
     if constexpr (POST && (MASK & SYNC_U)) {
         const float mu = mean_of<MT>(un);
@@ -168,13 +198,7 @@ __device__ __forceinline__ void update_coord(const StepArgs &a, const float (&g)
 #pragma unroll
     for (int m = 0; m < MT; ++m) {
         const float xp = (PRE && (MASK & SYNC_X)) ? xb : x[m];
-        float d;
-        if constexpr (OPT == OPT_ADAM)
-            d = (a.lr * un[m]) / sqrtf(vn[m] + a.lam2);
-        else
-            d = a.lr * un[m];
-        // x* (1 - eta wd) - d, written as x* - (eta wd x* + d): one rounding at x's scale
-        xn[m] = xp - fmaf(a.lrwd, xp, d);
+        xn[m] = param_step<OPT>(a, xp, un[m], vn[m]);
     }
     if constexpr (POST && (MASK & SYNC_X)) {
         const float mx = mean_of<MT>(xn);
@@ -189,12 +213,86 @@ __device__ __forceinline__ void update_coord(const StepArgs &a, const float (&g)
     }
 }
 
+// ---- pre-average tile for many workers: means first, then workers in batches -------------
+// With more than four replicas per thread the all-at-once tile needs more registers than two
+// resident blocks allow.  Here the arrays to be averaged are loaded for all MT workers and
+// reduced to their means; the per-worker phase then runs over batches of up to four workers,
+// loading only what is not averaged (ADOPT also its own v).  Same loads, same arithmetic, same
+// summation tree -- bitwise the same result as process_tile.
+template <int VEC, int MT>
+__device__ __forceinline__ FV<VEC> mean_over_workers(char *const *bases, long long e) {
+    FV<VEC> S[MT];
+#pragma unroll
+    for (int m = 0; m < MT; ++m) S[m] = ld_f32<VEC>(bases[m], e);
+    FV<VEC> r;
+#pragma unroll
+    for (int c = 0; c < VEC; ++c) {
+        float s[MT];
+#pragma unroll
+        for (int m = 0; m < MT; ++m) s[m] = S[m].a[c];
+        r.a[c] = mean_of<MT>(s);
+    }
+    return r;
+}
+
+template <int OPT, int MASK, int MT, typename GT, int VEC, int M0, int B>
+__device__ __forceinline__ void worker_batch(const StepArgs &a, char *const (*sp)[MT], long long e,
+                                             const FV<VEC> &xb, const FV<VEC> &ub,
+                                             const FV<VEC> &vb) {
+    constexpr bool SX = MASK & SYNC_X, SU = MASK & SYNC_U;
+    constexpr bool SV = (MASK & SYNC_V) && OPT != OPT_SGDM;
+    constexpr bool NEED_V = OPT != OPT_SGDM && (!SV || OPT == OPT_ADOPT);
+    FV<VEC> G[B], X[B], U[B], V[B];
+#pragma unroll
+    for (int b = 0; b < B; ++b) {
+        G[b] = ld_grad<VEC, GT>(sp[3][M0 + b], e);
+        if constexpr (!SX) X[b] = ld_f32<VEC>(sp[0][M0 + b], e);
+        if constexpr (!SU) U[b] = ld_f32<VEC>(sp[1][M0 + b], e);
+        if constexpr (NEED_V) V[b] = ld_f32<VEC>(sp[2][M0 + b], e);
+    }
+#pragma unroll
+    for (int b = 0; b < B; ++b) {
+#pragma unroll
+        for (int c = 0; c < VEC; ++c) {
+            const float up = SU ? ub.a[c] : U[b].a[c];
+            const float vown = NEED_V ? V[b].a[c] : 0.f;
+            const float vp = SV ? vb.a[c] : vown;
+            const float xp = SX ? xb.a[c] : X[b].a[c];
+            float un, vn;
+            state_update<OPT>(a, G[b].a[c], up, vp, vown, un, vn);
+            X[b].a[c] = param_step<OPT>(a, xp, un, vn);
+            U[b].a[c] = un;
+            V[b].a[c] = vn;
+        }
+        st_f32<VEC>(sp[0][M0 + b], e, X[b]);
+        st_f32<VEC>(sp[1][M0 + b], e, U[b]);
+        if constexpr (OPT != OPT_SGDM) st_f32<VEC>(sp[2][M0 + b], e, V[b]);
+    }
+}
+
+template <int OPT, int MASK, int MT, typename GT, int VEC>
+__device__ __forceinline__ void process_tile_split(const StepArgs &a, char *const (*sp)[MT],
+                                                   long long e) {
+    FV<VEC> xb{}, ub{}, vb{};
+    if constexpr (MASK & SYNC_X) xb = mean_over_workers<VEC, MT>(sp[0], e);
+    if constexpr (MASK & SYNC_U) ub = mean_over_workers<VEC, MT>(sp[1], e);
+    if constexpr ((MASK & SYNC_V) && OPT != OPT_SGDM) vb = mean_over_workers<VEC, MT>(sp[2], e);
+    worker_batch<OPT, MASK, MT, GT, VEC, 0, 4>(a, sp, e, xb, ub, vb);
+    worker_batch<OPT, MASK, MT, GT, VEC, 4, MT - 4>(a, sp, e, xb, ub, vb);
+}
+
 // ---- one thread's tile: MT workers x UN positions of VEC elements ------------------------
 // sp[arr][m] are chunk-relative base pointers in shared memory (arr: 0 x, 1 u, 2 v, 3 g).
 // Position j covers elements e0 + j * pstride .. + VEC - 1; positions >= npos are skipped.
 template <int OPT, int MASK, int MT, typename GT, bool POST, int VEC, int UN, bool FULL>
 __device__ __forceinline__ void process_tile(const StepArgs &a, char *const (*sp)[MT],
                                              long long e0, int pstride, int npos) {
+#if DESLOC_SPLIT_LARGE_M
+    if constexpr (!POST && MT > 4 && UN == 1 && OPT != OPT_SGDM) {
+        if (FULL || npos > 0) process_tile_split<OPT, MASK, MT, GT, VEC>(a, sp, e0);
+        return;
+    }
+#endif
     FV<VEC> G[UN][MT], X[UN][MT], U[UN][MT], V[UN][MT];
 #pragma unroll
     for (int j = 0; j < UN; ++j) {
@@ -241,22 +339,54 @@ __device__ __forceinline__ void process_tile(const StepArgs &a, char *const (*sp
     }
 }
 
+// Positions per thread and tile: one.  (Two positions for MT = 2 spilled under the register
+// cap of three blocks per SM; one worker at a time, MT = 1, only occurs on the ragged path of
+// desloc_local_kernel, which must stay light on registers next to the fast path.)
 template <int MT>
 struct UnrollFor {
-    static constexpr int value = MT == 1 ? 4 : (MT == 2 ? 2 : 1);
+    static constexpr int value = 1;
 };
 
+// One chunk of `count` elements for all MT workers: 128-bit path (with a scalar tail) when
+// every pointer is aligned, scalar path otherwise.
 template <int OPT, int MASK, int MT, typename GT, bool POST>
-__global__ void __launch_bounds__(BLOCK_THREADS, (MT <= 4 ? 3 : 2))
-desloc_step_kernel(const __grid_constant__ StepArgs a) {
+__device__ __forceinline__ void process_chunk(const StepArgs &a, char *const (*sp)[MT], int count,
+                                              bool scalar_path) {
     constexpr int UN = UnrollFor<MT>::value;
+    const int tid = threadIdx.x;
+    if (!scalar_path) {
+        if (count == CHUNK_ELEMS) {
+            // full chunk: 4 * UN * 256 * (4 / UN) elements, no bounds checks
+#pragma unroll 1
+            for (int r = 0; r < 4 / UN; ++r)
+                process_tile<OPT, MASK, MT, GT, POST, 4, UN, true>(
+                    a, sp, static_cast<long long>(r * UN * BLOCK_THREADS + tid) * 4,
+                    BLOCK_THREADS * 4, UN);
+        } else {
+            const int n4 = count >> 2;
+            for (int p0 = tid; p0 < n4; p0 += UN * BLOCK_THREADS) {
+                const int left = (n4 - p0 + BLOCK_THREADS - 1) / BLOCK_THREADS;
+                process_tile<OPT, MASK, MT, GT, POST, 4, UN, false>(
+                    a, sp, static_cast<long long>(p0) * 4, BLOCK_THREADS * 4,
+                    left < UN ? left : UN);
+            }
+            const int rem = count & 3;
+            if (tid < rem)
+                process_tile<OPT, MASK, MT, GT, POST, 1, 1, true>(a, sp, (n4 << 2) + tid, 0, 1);
+        }
+    } else {
+        for (int e = tid; e < count; e += BLOCK_THREADS)
+            process_tile<OPT, MASK, MT, GT, POST, 1, 1, true>(a, sp, e, 0, 1);
+    }
+}
+
+template <int OPT, int MASK, int MT, typename GT, bool POST>
+__global__ void __launch_bounds__(BLOCK_THREADS, (MT <= 4 ? 3 : ((OPT == OPT_SGDM || POST) ? 2 : DESLOC_MINB_LARGE_M)))
+desloc_step_kernel(const __grid_constant__ StepArgs a) {
     __shared__ char *sp[4][MT];
     const int tid = threadIdx.x;
-    // MT == 1 serves local steps of any M: item = (worker, chunk), workers independent.
-    const long long nitems = (MT == 1) ? a.nchunks * a.M : a.nchunks;
-    for (long long item = blockIdx.x; item < nitems; item += gridDim.x) {
-        const long long c = (MT == 1) ? item % a.nchunks : item;
-        const int m0 = (MT == 1) ? static_cast<int>(item / a.nchunks) : 0;
+    for (long long c = blockIdx.x; c < a.nchunks; c += gridDim.x) {
+        constexpr int m0 = 0;
         const Chunk ch = a.chunks[c];
         __syncthreads();  // previous chunk's readers are done with sp
         int misaligned = 0;
@@ -275,34 +405,76 @@ desloc_step_kernel(const __grid_constant__ StepArgs a) {
             misaligned = (reinterpret_cast<uintptr_t>(p) & need) != 0;
         }
         const int scalar_path = __syncthreads_or(misaligned);
-        if (!scalar_path) {
-            if (ch.count == CHUNK_ELEMS) {
-                // full chunk: 4 * UN * 256 * (4 / UN) elements, no bounds checks
-#pragma unroll 1
-                for (int r = 0; r < 4 / UN; ++r)
-                    process_tile<OPT, MASK, MT, GT, POST, 4, UN, true>(
-                        a, sp, static_cast<long long>(r * UN * BLOCK_THREADS + tid) * 4,
-                        BLOCK_THREADS * 4, UN);
-            } else {
-                const int n4 = ch.count >> 2;
-                for (int p0 = tid; p0 < n4; p0 += UN * BLOCK_THREADS) {
-                    const int left = (n4 - p0 + BLOCK_THREADS - 1) / BLOCK_THREADS;
-                    process_tile<OPT, MASK, MT, GT, POST, 4, UN, false>(
-                        a, sp, static_cast<long long>(p0) * 4, BLOCK_THREADS * 4,
-                        left < UN ? left : UN);
-                }
-                const int rem = ch.count & 3;
-                if (tid < rem)
-                    process_tile<OPT, MASK, MT, GT, POST, 1, 1, true>(a, sp, (n4 << 2) + tid, 0, 1);
+        process_chunk<OPT, MASK, MT, GT, POST>(a, sp, ch.count, scalar_path != 0);
+    }
+}
+
+// ---- local steps with workers as separate work items (M = 1, or M > MAX_MT) -------------
+// A block takes LOCAL_SLOTS consecutive chunks of one worker: their pointers are set up
+// together (one dependent-load chain instead of four) and, when all of them are full and
+// aligned, they are processed exactly like four replicas of one chunk on a local step.
+constexpr int LOCAL_SLOTS = 4;
+
+template <int OPT, typename GT>
+__global__ void __launch_bounds__(BLOCK_THREADS, 3)
+desloc_local_kernel(const __grid_constant__ StepArgs a) {
+    constexpr int SL = LOCAL_SLOTS;
+    __shared__ char *sp[4][SL];
+    __shared__ int scount[SL];
+    const int tid = threadIdx.x;
+    const long long ngroups = (a.nchunks + SL - 1) / SL;
+    const long long nitems = ngroups * a.M;
+    for (long long item = blockIdx.x; item < nitems; item += gridDim.x) {
+        const long long grp = item % ngroups;
+        const int m0 = static_cast<int>(item / ngroups);
+        __syncthreads();
+        int slow = 0;
+        if (tid < 4 * SL) {
+            const int arr = tid / SL, sl = tid - arr * SL;
+            const long long c = grp * SL + sl;
+            char *p = nullptr;
+            int cnt = 0;
+            if (c < a.nchunks) {
+                const Chunk ch = a.chunks[c];
+                cnt = ch.count;
+                const long long idx = static_cast<long long>(m0) * a.nt + ch.tensor;
+                if (arr == 0) p = reinterpret_cast<char *>(a.x[idx]) + ch.start * 4;
+                if (arr == 1) p = reinterpret_cast<char *>(a.u[idx]) + ch.start * 4;
+                if (arr == 2 && OPT != OPT_SGDM) p = reinterpret_cast<char *>(a.v[idx]) + ch.start * 4;
+                if (arr == 3)
+                    p = const_cast<char *>(reinterpret_cast<const char *>(a.g[idx])) +
+                        ch.start * static_cast<long long>(sizeof(GT));
             }
+            sp[arr][sl] = p;
+            if (arr == 0) scount[sl] = cnt;
+            const unsigned need = (arr == 3 && sizeof(GT) == 2) ? 7u : 15u;
+            slow = cnt != CHUNK_ELEMS || (reinterpret_cast<uintptr_t>(p) & need) != 0;
+        }
+        if (!__syncthreads_or(slow)) {
+#pragma unroll 1
+            for (int r = 0; r < 4; ++r)
+                process_tile<OPT, 0, SL, GT, false, 4, 1, true>(
+                    a, sp, static_cast<long long>(r * BLOCK_THREADS + tid) * 4, BLOCK_THREADS * 4, 1);
         } else {
-            for (int e = tid; e < ch.count; e += BLOCK_THREADS)
-                process_tile<OPT, MASK, MT, GT, POST, 1, 1, true>(a, sp, e, 0, 1);
+            // ragged group (a tensor's last chunk, an unaligned tensor, the list's end): slot by slot
+#pragma unroll 1
+            for (int sl = 0; sl < SL; ++sl) {
+                const int cnt = scount[sl];
+                if (cnt == 0) continue;
+                char *one[4][1] = {{sp[0][sl]}, {sp[1][sl]}, {sp[2][sl]}, {sp[3][sl]}};
+                unsigned long long bits = reinterpret_cast<uintptr_t>(one[0][0]) |
+                                          reinterpret_cast<uintptr_t>(one[1][0]) |
+                                          reinterpret_cast<uintptr_t>(one[2][0]);
+                const bool mis = (bits & 15u) != 0 ||
+                                 (reinterpret_cast<uintptr_t>(one[3][0]) & (sizeof(GT) == 2 ? 7u : 15u)) != 0;
+                process_chunk<OPT, 0, 1, GT, false>(a, one, cnt, mis);
+            }
         }
     }
 }
 
-// Lookup of an instantiation: opt, post-average?, bf16 gradients?, MT in 1..MAX_MT, mask.
+// Lookup of an instantiation: opt, post-average?, bf16 gradients?, MT in 1..MAX_MT, mask
+// (mt = 1 with mask 0 is desloc_local_kernel).
 // Returns nullptr for combinations that do not exist (sync masks with M > MAX_MT).
 const void *lookup_step_kernel(int opt, bool post, bool bf16, int mt, int mask);
 

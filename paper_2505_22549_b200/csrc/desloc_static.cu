@@ -163,7 +163,8 @@ extern "C" DESLOC_API int desloc_step_static(const desloc_config *cfg, float *co
         a.lrwd = static_cast<float>(static_cast<double>(lr_t) * static_cast<double>(cfg->weight_decay));
         a.rho = cfg->clip_rho > 0.f ? cfg->clip_rho : std::numeric_limits<float>::infinity();
         a.cbound = nclip ? clip_bound_t : std::numeric_limits<float>::infinity();
-        const long long nitems = (cfg->M == 1) ? nchunks * cfg->M : nchunks;
+        const long long nitems =
+            (cfg->M == 1) ? (nchunks + desloc::LOCAL_SLOTS - 1) / desloc::LOCAL_SLOTS : nchunks;
         void *params[] = {&a};
         e = cudaLaunchKernel(fn, dim3(static_cast<unsigned>(nitems)), dim3(desloc::BLOCK_THREADS),
                              params, 0, st);
