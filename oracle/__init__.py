@@ -68,6 +68,15 @@ def lib() -> ctypes.CDLL:
             ctypes.POINTER(OracleCfg), ctypes.c_int64, ctypes.c_double, ctypes.c_double,
             ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
             ctypes.c_void_p]
+        L.desloc_oracle_step_scaled.restype = ctypes.c_uint32
+        L.desloc_oracle_step_scaled.argtypes = L.desloc_oracle_step.argtypes + [ctypes.c_void_p]
+        L.desloc_oracle_norm_scales.restype = None
+        L.desloc_oracle_norm_scales.argtypes = [ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
+                                                ctypes.c_void_p, ctypes.c_double, ctypes.c_void_p,
+                                                ctypes.c_void_p]
+        L.desloc_oracle_rel_change.restype = None
+        L.desloc_oracle_rel_change.argtypes = [ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
+                                               ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         L.desloc_oracle_run.restype = None
         L.desloc_oracle_run.argtypes = [
             ctypes.POINTER(OracleCfg), ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p,
@@ -98,14 +107,42 @@ def _check(a, M, name, allow_none=False):
     return a.ctypes.data
 
 
-def step(cfg: OracleCfg, t: int, lr: float, x, u, v, g, clip_bound: float = 0.0) -> int:
-    """One step in place on float32 arrays of shape [M, n]; returns the sync mask."""
+def norm_scales(g, max_norm: float):
+    """Per-worker gradient norms and norm-clip factors min(1, max_norm/||g^m||) for g of shape [M, n]."""
+    M = g.shape[0]
+    pg = _check(g, M, "g")
+    norms = np.zeros(M, dtype=np.float64)
+    scales = np.zeros(M, dtype=np.float64)
+    lib().desloc_oracle_norm_scales(M, g.shape[1], g.shape[1], pg, float(max_norm),
+                                    norms.ctypes.data, scales.ctypes.data)
+    return norms, scales
+
+
+def rel_change(now, then):
+    """Per-worker ||now - then||_2 / ||then||_2 for float32 arrays of shape [M, n]."""
+    M = now.shape[0]
+    pn, pt = _check(now, M, "now"), _check(then, M, "then")
+    out = np.zeros(M, dtype=np.float64)
+    lib().desloc_oracle_rel_change(M, now.shape[1], now.shape[1], pn, pt, out.ctypes.data)
+    return out
+
+
+def step(cfg: OracleCfg, t: int, lr: float, x, u, v, g, clip_bound: float = 0.0,
+         gscale=None) -> int:
+    """One step in place on float32 arrays of shape [M, n]; returns the sync mask.
+    gscale: optional per-worker factors applied to g before the coordinate clip."""
     M = cfg.M
     px, pu, pg = _check(x, M, "x"), _check(u, M, "u"), _check(g, M, "g")
     pv = _check(v, M, "v", allow_none=(cfg.opt == SGDM))
     n = x.shape[1]
     if u.shape != x.shape or g.shape != x.shape or (v is not None and v.shape != x.shape):
         raise ValueError("x, u, v, g must share one shape")
+    if gscale is not None:
+        gs = np.ascontiguousarray(gscale, dtype=np.float64)
+        assert gs.shape == (M,)
+        return int(lib().desloc_oracle_step_scaled(ctypes.byref(cfg), int(t), float(lr),
+                                                   float(clip_bound), n, n, px, pu, pv, pg,
+                                                   gs.ctypes.data))
     return int(lib().desloc_oracle_step(ctypes.byref(cfg), int(t), float(lr), float(clip_bound),
                                         n, n, px, pu, pv, pg))
 

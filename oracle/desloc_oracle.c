@@ -35,6 +35,10 @@
  *   - no bias-correction factor is applied: none appears in Algorithm 2's
  *     formulas.  A caller folds it into eta_t.
  *
+ *   - norm-based clipping (used by the paper's language-model runs, absent from the
+ *     algorithm listings) scales each worker's whole gradient by min(1, rho_norm/||g||_2)
+ *     BEFORE the coordinate clip; no epsilon is added to the norm.
+ *
  * Pins (tests/test_oracle_pins.py): M=1 against torch.optim.Adam / AdamW / SGD
  * in fp64; identical gradients keep replicas equal to the single-worker run;
  * the worker-mean of u, v (and of x for SGDM) does not depend on the schedule;
@@ -98,9 +102,9 @@ static double worker_mean(const float *s, int64_t stride, int64_t i, int M) {
  * (worker-major), g already widened to fp32 (bf16 widens exactly).  v may be
  * NULL for SGDM.  Updates x, u, v in place; returns the sync mask used.
  */
-uint32_t desloc_oracle_step(const desloc_oracle_cfg *c, int64_t t, double lr, double clip_bound,
-                            int64_t n, int64_t stride, float *x, float *u, float *v,
-                            const float *g) {
+uint32_t desloc_oracle_step_scaled(const desloc_oracle_cfg *c, int64_t t, double lr,
+                                   double clip_bound, int64_t n, int64_t stride, float *x, float *u,
+                                   float *v, const float *g, const double *gscale) {
     const int M = c->M;
     const uint32_t mask = desloc_oracle_sync_mask(c->opt, c->Kx, c->Ku, c->Kv, t);
     const int post = (c->flags & DESLOC_ORACLE_POST_AVERAGE) != 0;
@@ -119,7 +123,8 @@ uint32_t desloc_oracle_step(const desloc_oracle_cfg *c, int64_t t, double lr, do
         /* ---- optimizer states ------------------------------------------- */
         for (int m = 0; m < M; ++m) {
             const int64_t k = (int64_t)m * stride + i;
-            const double gh = clip_coord((double)g[k], c->clip_rho);
+            const double gs = gscale ? gscale[m] : 1.0; /* norm-based clip factor, if any */
+            const double gh = clip_coord((double)g[k] * gs, c->clip_rho);
             const double up = (!post && (mask & ORACLE_SYNC_U)) ? ubar : (double)u[k];
             double vp = 0.0;
             if (c->opt != ORACLE_SGDM)
@@ -194,6 +199,50 @@ uint32_t desloc_oracle_step(const desloc_oracle_cfg *c, int64_t t, double lr, do
     free(un);
     free(vn);
     return mask;
+}
+
+uint32_t desloc_oracle_step(const desloc_oracle_cfg *c, int64_t t, double lr, double clip_bound,
+                            int64_t n, int64_t stride, float *x, float *u, float *v,
+                            const float *g) {
+    return desloc_oracle_step_scaled(c, t, lr, clip_bound, n, stride, x, u, v, g, NULL);
+}
+
+/*
+ * Norm-based gradient clipping, the form the paper's language-model runs used (model table:
+ * "norm-based gradient clipping with clip-bound rho"): worker m's whole gradient (all tensors,
+ * here one [M][stride] array) is scaled by min(1, max_norm / ||g^m||_2).  Writes the norms and
+ * the factors; a zero gradient keeps factor 1.
+ */
+void desloc_oracle_norm_scales(int32_t M, int64_t n, int64_t stride, const float *g, double max_norm,
+                               double *norms_out, double *scales_out) {
+    for (int m = 0; m < M; ++m) {
+        double acc = 0.0;
+        for (int64_t i = 0; i < n; ++i) {
+            const double a = (double)g[(int64_t)m * stride + i];
+            acc += a * a;
+        }
+        const double nrm = sqrt(acc);
+        norms_out[m] = nrm;
+        scales_out[m] = (nrm > max_norm) ? max_norm / nrm : 1.0;
+    }
+}
+
+/*
+ * Relative change of a state over an interval, ||s_now - s_then||_2 / ||s_then||_2 per worker
+ * (the rate-of-change measure of Section 5.1, "Metrics").
+ */
+void desloc_oracle_rel_change(int32_t M, int64_t n, int64_t stride, const float *now,
+                              const float *then, double *out) {
+    for (int m = 0; m < M; ++m) {
+        double num = 0.0, den = 0.0;
+        for (int64_t i = 0; i < n; ++i) {
+            const double a = (double)now[(int64_t)m * stride + i];
+            const double b = (double)then[(int64_t)m * stride + i];
+            num += (a - b) * (a - b);
+            den += b * b;
+        }
+        out[m] = sqrt(num) / sqrt(den);
+    }
 }
 
 /*

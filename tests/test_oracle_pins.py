@@ -507,3 +507,47 @@ def test_post_average_equals_pre_average_shifted_by_one_step(opt):
         assert np.array_equal(a_post[0], a_post[1]) and np.array_equal(a_post[1], a_post[2])
     if opt == ADAM:
         assert not np.allclose(_mean(res[False][0]), res[True][0][0].astype(np.float64), rtol=1e-7, atol=0)
+
+
+# --------------------------------------------------------------------------- norm-based clipping
+def test_norm_scales_match_torch_clip_grad_norm():
+    """Library routine: torch.nn.utils.clip_grad_norm_ scales by max_norm / (norm + 1e-6) (clamped
+    to 1); the oracle by max_norm / norm.  They agree to that epsilon."""
+    rng = np.random.default_rng(11)
+    sizes = [7, 130, 1, 64]
+    for scale, max_norm in [(1.0, 1.0), (1e-3, 1.0), (5.0, 0.25)]:
+        tensors = [rng.normal(size=s).astype(np.float32) * scale for s in sizes]
+        params = [torch.nn.Parameter(torch.zeros(s, dtype=torch.float64)) for s in sizes]
+        for p, t in zip(params, tensors):
+            p.grad = torch.tensor(t, dtype=torch.float64)
+        total = float(torch.nn.utils.clip_grad_norm_(params, max_norm))
+        flat = f32(np.concatenate(tensors)[None])
+        norms, scales = oracle.norm_scales(flat, max_norm)
+        assert abs(norms[0] - total) <= 1e-12 * total
+        clipped = np.concatenate([p.grad.numpy() for p in params])
+        assert np.allclose(flat[0].astype(np.float64) * scales[0], clipped, rtol=3e-6, atol=0)
+        if total <= max_norm:
+            assert scales[0] == 1.0
+
+
+def test_norm_clip_closed_forms():
+    g = f32([[3.0, 4.0, 0.0], [0.3, 0.4, 0.0], [0.0, 0.0, 0.0]])      # norms 5, 0.5, 0
+    norms, scales = oracle.norm_scales(g, 1.0)
+    assert np.allclose(norms, [5.0, 0.5, 0.0], rtol=1e-7)
+    assert np.allclose(scales, [0.2, 1.0, 1.0], rtol=1e-7)
+    # after scaling the norm is min(norm, max_norm)
+    assert abs(np.linalg.norm(g[0].astype(np.float64) * scales[0]) - 1.0) < 1e-7
+    # the scaled gradient feeds the coordinate clip and the update: SGDM, beta = 0 -> u = clip(s*g)
+    cfg = oracle.make_cfg(3, SGDM, beta1=0.0, clip_rho=0.5, Kx=0, Ku=0, Kv=0)
+    x, u = zeros(3, 3), zeros(3, 3)
+    oracle.step(cfg, 0, 1.0, x, u, None, g, gscale=scales)
+    assert np.allclose(u, [[0.5, 0.5, 0.0], [0.3, 0.4, 0.0], [0.0, 0.0, 0.0]], rtol=1e-6)
+
+
+def test_rel_change_closed_forms():
+    then = f32([[1.0, 2.0, 2.0], [3.0, 0.0, 4.0]])
+    now = f32([[2.0, 4.0, 4.0], [3.0, 0.0, 4.0]])
+    out = oracle.rel_change(now, then)
+    assert np.allclose(out, [1.0, 0.0])
+    now2 = f32([[1.0, 2.0, 5.0], [0.0, 0.0, 0.0]])      # diff (0,0,3)/3 ; (3,0,4)/5
+    assert np.allclose(oracle.rel_change(now2, then), [1.0, 1.0])
