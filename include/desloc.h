@@ -138,6 +138,38 @@ DESLOC_API int desloc_step(desloc_ctx *ctx, int64_t t, float lr_t, float clip_bo
 DESLOC_API int desloc_step_masked(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
                        const void *const *grads, void *stream);
 
+/*
+ * One step with norm-based gradient clipping in front: worker m's whole gradient (all tensors)
+ * is scaled by min(1, max_norm / ||g^m||_2) before the coordinate clip and the update.  This
+ * is the clipping the paper's language-model runs used (model table in the experimental
+ * details: "norm-based gradient clipping with clip-bound rho", rho = 1.0); Algorithms 1-3
+ * only have the coordinate-wise clip.  Costs one more read of the gradients: two reduction
+ * launches (per-chunk partial sums in fp32, per-worker totals in fp64, fixed order, no
+ * atomics) ahead of the step kernel, all enqueued on `stream` without host synchronisation.
+ * max_norm must be > 0 and finite.  Other arguments as desloc_step().
+ */
+DESLOC_API int desloc_step_normclip(desloc_ctx *ctx, int64_t t, float lr_t, float clip_bound_t,
+                                    float max_norm, const void *const *grads, void *stream,
+                                    uint32_t *mask_out);
+
+/*
+ * Gradient norms ||g^m||_2 and clip factors of the latest desloc_step_normclip() into the host
+ * arrays norms_out[M], scales_out[M] (either may be NULL).  Copies on `stream` and waits for
+ * it: this call synchronises.
+ */
+DESLOC_API int desloc_get_grad_norms(desloc_ctx *ctx, float *norms_out, float *scales_out,
+                                     void *stream);
+
+/*
+ * Relative change of a state since a snapshot, per worker: out[m] = ||s^m - then^m||_2 /
+ * ||then^m||_2 over the whole tensor list (the rate-of-change measure of Section 5.1,
+ * "Metrics", ||s_{t+K} - s_t|| / ||s_t||).  array: 0 = x, 1 = u, 2 = v.  then: host array of
+ * M*num_tensors DEVICE pointers to the caller's fp32 snapshot (same shapes as the state).
+ * out: host array [M].  Enqueues on `stream` and waits for it: this call synchronises.
+ */
+DESLOC_API int desloc_rel_change(desloc_ctx *ctx, int32_t array, const float *const *then,
+                                 float *out, void *stream);
+
 /* Release the context and everything it allocated.  The caller's tensors are untouched.
    NULL is a no-op returning DESLOC_OK. */
 DESLOC_API int desloc_destroy(desloc_ctx *ctx);

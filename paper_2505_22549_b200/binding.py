@@ -78,6 +78,14 @@ _lib.desloc_step_masked.restype = ctypes.c_int
 _lib.desloc_step_masked.argtypes = [_P, ctypes.c_uint32, ctypes.c_float, ctypes.c_float, _PP, _P]
 _lib.desloc_destroy.restype = ctypes.c_int
 _lib.desloc_destroy.argtypes = [_P]
+_lib.desloc_step_normclip.restype = ctypes.c_int
+_lib.desloc_step_normclip.argtypes = [_P, ctypes.c_int64, ctypes.c_float, ctypes.c_float,
+                                      ctypes.c_float, _PP, _P, ctypes.POINTER(ctypes.c_uint32)]
+_lib.desloc_get_grad_norms.restype = ctypes.c_int
+_lib.desloc_get_grad_norms.argtypes = [_P, ctypes.POINTER(ctypes.c_float),
+                                       ctypes.POINTER(ctypes.c_float), _P]
+_lib.desloc_rel_change.restype = ctypes.c_int
+_lib.desloc_rel_change.argtypes = [_P, ctypes.c_int32, _PP, ctypes.POINTER(ctypes.c_float), _P]
 _lib.desloc_step_static.restype = ctypes.c_int
 _lib.desloc_step_static.argtypes = [ctypes.POINTER(DeslocConfig), _PP, _PP, _PP, _PP,
                                     ctypes.c_int64, ctypes.c_float, ctypes.c_float, ctypes.c_int,
@@ -179,6 +187,36 @@ def desloc_step_static(cfg: DeslocConfig, x, u, v, grads, t: int, lr_t: float,
     if rc != DESLOC_OK:
         raise DeslocError(rc, "desloc_step_static")
     return int(mask.value)
+
+
+def desloc_step_normclip(ctx: int, t: int, lr_t: float, clip_bound_t: float, max_norm: float,
+                         grads, stream: int = 0) -> int:
+    """One step with norm-based gradient clipping in front; returns the sync mask."""
+    g = grads if isinstance(grads, ctypes.Array) else _ptr_array(grads)
+    mask = ctypes.c_uint32(0)
+    rc = _lib.desloc_step_normclip(ctx, int(t), float(lr_t), float(clip_bound_t), float(max_norm),
+                                   g, stream or None, ctypes.byref(mask))
+    if rc != DESLOC_OK:
+        raise DeslocError(rc, "desloc_step_normclip", _lib.desloc_last_cuda_error(ctx))
+    return int(mask.value)
+
+
+def desloc_get_grad_norms(ctx: int, M: int, stream: int = 0):
+    """(norms, clip factors) of the latest desloc_step_normclip as two lists of M floats."""
+    norms, scales = (ctypes.c_float * M)(), (ctypes.c_float * M)()
+    rc = _lib.desloc_get_grad_norms(ctx, norms, scales, stream or None)
+    if rc != DESLOC_OK:
+        raise DeslocError(rc, "desloc_get_grad_norms", _lib.desloc_last_cuda_error(ctx))
+    return list(norms), list(scales)
+
+
+def desloc_rel_change(ctx: int, array: int, then: Sequence[int], M: int, stream: int = 0):
+    """Per-worker ||s - then|| / ||then|| for array 0 = x, 1 = u, 2 = v; `then` are device pointers."""
+    out = (ctypes.c_float * M)()
+    rc = _lib.desloc_rel_change(ctx, int(array), _ptr_array(then), out, stream or None)
+    if rc != DESLOC_OK:
+        raise DeslocError(rc, "desloc_rel_change", _lib.desloc_last_cuda_error(ctx))
+    return list(out)
 
 
 def desloc_destroy(ctx: Optional[int]) -> None:

@@ -71,7 +71,12 @@ __device__ __forceinline__ void generic_position(const StepArgs &a, const Chunk 
         const FV<VEC> xb = acc_mean<VEC>(ax, M), ub = acc_mean<VEC>(au, M), vb = acc_mean<VEC>(av, M);
         for (int m = 0; m < M; ++m) {
             const Ptrs p = worker_ptrs<OPT, GT>(a, ch, m);
-            const FV<VEC> G = ld_grad<VEC, GT>(p.g, e);
+            FV<VEC> G = ld_grad<VEC, GT>(p.g, e);
+            if (a.gscale) {
+                const float sc = a.gscale[m];
+#pragma unroll
+                for (int c = 0; c < VEC; ++c) G.a[c] *= sc;
+            }
             FV<VEC> X = sx ? xb : ld_f32<VEC>(p.x, e);
             FV<VEC> U = su ? ub : ld_f32<VEC>(p.u, e);
             FV<VEC> V{}, Vown{};
@@ -108,7 +113,12 @@ __device__ __forceinline__ void generic_position(const StepArgs &a, const Chunk 
         double au[VEC] = {}, av[VEC] = {}, ax[VEC] = {};
         for (int m = 0; m < M; ++m) {
             const Ptrs p = worker_ptrs<OPT, GT>(a, ch, m);
-            const FV<VEC> G = ld_grad<VEC, GT>(p.g, e);
+            FV<VEC> G = ld_grad<VEC, GT>(p.g, e);
+            if (a.gscale) {
+                const float sc = a.gscale[m];
+#pragma unroll
+                for (int c = 0; c < VEC; ++c) G.a[c] *= sc;
+            }
             FV<VEC> U = ld_f32<VEC>(p.u, e), V{};
             if constexpr (OPT != OPT_SGDM) V = ld_f32<VEC>(p.v, e);
 #pragma unroll

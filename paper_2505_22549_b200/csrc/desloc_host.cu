@@ -13,6 +13,7 @@
 
 #include "../../include/desloc.h"
 #include "desloc_inst.cuh"
+#include "desloc_norms.cuh"
 
 namespace desloc {
 
@@ -67,6 +68,11 @@ struct desloc_ctx {
     int64_t launches = 0;
     int last_cuda_error = 0;
     int ctas_per_sm = 0;  // 0: one block per work item; > 0: persistent grid of that many per SM
+    // reductions: partial sums [2][M][nchunks], per-worker norms / clip factors / rel. change
+    float *d_partial = nullptr;
+    float *d_norms = nullptr;   // [3][M]: norms, scales, relative change
+    void **h_snap = nullptr;    // pinned pointer table for desloc_rel_change
+    void **d_snap = nullptr;
 };
 
 namespace {
@@ -116,6 +122,10 @@ void free_ctx(desloc_ctx *ctx) {
         if (s.host) cudaFreeHost(s.host);
         if (s.dev) cudaFree(s.dev);
     }
+    if (ctx->d_partial) cudaFree(ctx->d_partial);
+    if (ctx->d_norms) cudaFree(ctx->d_norms);
+    if (ctx->h_snap) cudaFreeHost(ctx->h_snap);
+    if (ctx->d_snap) cudaFree(ctx->d_snap);
     if (ctx->d_chunks) cudaFree(ctx->d_chunks);
     if (ctx->d_tables) cudaFree(ctx->d_tables);
     delete ctx;
@@ -147,10 +157,11 @@ int stage_grads(desloc_ctx *ctx, const void *const *grads, cudaStream_t stream, 
     return DESLOC_OK;
 }
 
+// max_norm > 0: norm-based clipping first (two reduction launches), then the step.
 int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
-             const void *const *grads, cudaStream_t stream) {
+             const void *const *grads, cudaStream_t stream, float max_norm = 0.f) {
     const desloc_config &c = ctx->cfg;
-    if (!std::isfinite(lr_t)) return DESLOC_E_RANGE;
+    if (!std::isfinite(lr_t) || std::isnan(max_norm)) return DESLOC_E_RANGE;
     const bool nclip = (c.flags & DESLOC_FLAG_ADOPT_NORM_CLIP) != 0;
     if (nclip && !(clip_bound_t >= 0.f)) return DESLOC_E_RANGE;
     for (int64_t i = 0; i < ctx->nptr; ++i)
@@ -168,6 +179,20 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
         void **d_g = nullptr;
         rc = stage_grads(ctx, grads, stream, &d_g);
         if (rc != DESLOC_OK) break;
+
+        const float *d_gscale = nullptr;
+        if (max_norm > 0.f) {
+            e = desloc::launch_grad_norms(ctx->d_chunks, ctx->nchunks,
+                                          reinterpret_cast<const void *const *>(d_g), c.num_tensors,
+                                          c.M, c.grad_dtype == DESLOC_BF16, max_norm,
+                                          ctx->d_partial, ctx->d_norms, ctx->d_norms + c.M, stream);
+            if (e != cudaSuccess) {
+                rc = cuda_fail(ctx, e);
+                break;
+            }
+            ctx->launches += 2;
+            d_gscale = ctx->d_norms + c.M;
+        }
 
         // The mean of one replica is the replica: M = 1 always runs the local kernel.
         const uint32_t kmask = (c.M == 1) ? 0u : mask;
@@ -189,6 +214,7 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
         a.u = reinterpret_cast<float *const *>(ctx->d_tables + ctx->nptr);
         a.v = reinterpret_cast<float *const *>(ctx->d_tables + 2 * ctx->nptr);
         a.g = reinterpret_cast<const void *const *>(d_g);
+        a.gscale = d_gscale;
         a.nt = c.num_tensors;
         a.M = c.M;
         a.b1 = c.beta1;
@@ -334,6 +360,12 @@ int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *const *x, f
     if (e == cudaSuccess)
         e = cudaMemcpy(ctx->d_tables, tables.data(), tables.size() * sizeof(void *),
                        cudaMemcpyHostToDevice);
+    const size_t npart = static_cast<size_t>(2) * cfg->M * chunks.size();
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_partial, npart * sizeof(float));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_norms, static_cast<size_t>(3) * cfg->M * sizeof(float));
+    if (e == cudaSuccess) e = cudaMemset(ctx->d_norms, 0, static_cast<size_t>(3) * cfg->M * sizeof(float));
+    if (e == cudaSuccess) e = cudaMallocHost(&ctx->h_snap, static_cast<size_t>(nptr) * sizeof(void *));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_snap, static_cast<size_t>(nptr) * sizeof(void *));
     for (int i = 0; i < kSlots && e == cudaSuccess; ++i) {
         Slot &s = ctx->slots[i];
         e = cudaMallocHost(&s.host, static_cast<size_t>(nptr) * sizeof(void *));
@@ -366,6 +398,62 @@ int desloc_step_masked(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bo
     if (mask & ~7u) return DESLOC_E_INVALID;
     if (ctx->cfg.opt == DESLOC_SGDM && (mask & DESLOC_SYNC_V)) return DESLOC_E_INVALID;
     return run_step(ctx, mask, lr_t, clip_bound_t, grads, static_cast<cudaStream_t>(stream));
+}
+
+int desloc_step_normclip(desloc_ctx *ctx, int64_t t, float lr_t, float clip_bound_t,
+                         float max_norm, const void *const *grads, void *stream,
+                         uint32_t *mask_out) {
+    if (!ctx || !grads) return DESLOC_E_NULL;
+    if (t < 0 || !(max_norm > 0.f) || !std::isfinite(max_norm)) return DESLOC_E_RANGE;
+    const uint32_t mask = mask_at(&ctx->cfg, t);
+    const int rc = run_step(ctx, mask, lr_t, clip_bound_t, grads, static_cast<cudaStream_t>(stream),
+                            max_norm);
+    if (rc == DESLOC_OK && mask_out) *mask_out = mask;
+    return rc;
+}
+
+int desloc_get_grad_norms(desloc_ctx *ctx, float *norms_out, float *scales_out, void *stream) {
+    if (!ctx) return DESLOC_E_NULL;
+    const size_t bytes = static_cast<size_t>(ctx->cfg.M) * sizeof(float);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaSuccess;
+    if (norms_out) e = cudaMemcpyAsync(norms_out, ctx->d_norms, bytes, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess && scales_out)
+        e = cudaMemcpyAsync(scales_out, ctx->d_norms + ctx->cfg.M, bytes, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    return e == cudaSuccess ? DESLOC_OK : cuda_fail(ctx, e);
+}
+
+int desloc_rel_change(desloc_ctx *ctx, int32_t array, const float *const *then, float *out,
+                      void *stream) {
+    if (!ctx || !then || !out) return DESLOC_E_NULL;
+    if (array < 0 || array > 2 || (array == 2 && ctx->cfg.opt == DESLOC_SGDM)) return DESLOC_E_INVALID;
+    for (int64_t i = 0; i < ctx->nptr; ++i)
+        if (!then[i]) return DESLOC_E_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int dev_before = -1;
+    cudaError_t e = cudaGetDevice(&dev_before);
+    if (e == cudaSuccess && dev_before != ctx->device) e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    const size_t tbytes = static_cast<size_t>(ctx->nptr) * sizeof(void *);
+    // The call ends with a stream synchronisation, so the pinned table is free again on return.
+    std::memcpy(ctx->h_snap, then, tbytes);
+    e = cudaMemcpyAsync(ctx->d_snap, ctx->h_snap, tbytes, cudaMemcpyHostToDevice, st);
+    float *d_out = ctx->d_norms + 2 * ctx->cfg.M;
+    if (e == cudaSuccess)
+        e = desloc::launch_rel_change(
+            ctx->d_chunks, ctx->nchunks,
+            reinterpret_cast<const float *const *>(ctx->d_tables + array * ctx->nptr),
+            reinterpret_cast<const float *const *>(ctx->d_snap), ctx->cfg.num_tensors, ctx->cfg.M,
+            ctx->d_partial, d_out, st);
+    if (e == cudaSuccess) {
+        ctx->launches += 2;
+        e = cudaMemcpyAsync(out, d_out, static_cast<size_t>(ctx->cfg.M) * sizeof(float),
+                            cudaMemcpyDeviceToHost, st);
+    }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (dev_before != ctx->device) cudaSetDevice(dev_before);
+    return e == cudaSuccess ? DESLOC_OK : cuda_fail(ctx, e);
 }
 
 int desloc_destroy(desloc_ctx *ctx) {

@@ -49,6 +49,7 @@ struct StepArgs {
     float *const *u;
     float *const *v;
     const void *const *g;
+    const float *gscale;  // per-worker factor applied to g before the clip, or nullptr (= 1)
     int nt;
     int M;
     float b1, omb1;   // beta1, 1 - beta1
@@ -236,7 +237,8 @@ __device__ __forceinline__ FV<VEC> mean_over_workers(char *const *bases, long lo
 }
 
 template <int OPT, int MASK, int MT, typename GT, int VEC, int M0, int B>
-__device__ __forceinline__ void worker_batch(const StepArgs &a, char *const (*sp)[MT], long long e,
+__device__ __forceinline__ void worker_batch(const StepArgs &a, char *const (*sp)[MT],
+                                             const float *sscale, long long e,
                                              const FV<VEC> &xb, const FV<VEC> &ub,
                                              const FV<VEC> &vb) {
     constexpr bool SX = MASK & SYNC_X, SU = MASK & SYNC_U;
@@ -259,7 +261,7 @@ __device__ __forceinline__ void worker_batch(const StepArgs &a, char *const (*sp
             const float vp = SV ? vb.a[c] : vown;
             const float xp = SX ? xb.a[c] : X[b].a[c];
             float un, vn;
-            state_update<OPT>(a, G[b].a[c], up, vp, vown, un, vn);
+            state_update<OPT>(a, G[b].a[c] * sscale[M0 + b], up, vp, vown, un, vn);
             X[b].a[c] = param_step<OPT>(a, xp, un, vn);
             U[b].a[c] = un;
             V[b].a[c] = vn;
@@ -272,13 +274,13 @@ __device__ __forceinline__ void worker_batch(const StepArgs &a, char *const (*sp
 
 template <int OPT, int MASK, int MT, typename GT, int VEC>
 __device__ __forceinline__ void process_tile_split(const StepArgs &a, char *const (*sp)[MT],
-                                                   long long e) {
+                                                   const float *sscale, long long e) {
     FV<VEC> xb{}, ub{}, vb{};
     if constexpr (MASK & SYNC_X) xb = mean_over_workers<VEC, MT>(sp[0], e);
     if constexpr (MASK & SYNC_U) ub = mean_over_workers<VEC, MT>(sp[1], e);
     if constexpr ((MASK & SYNC_V) && OPT != OPT_SGDM) vb = mean_over_workers<VEC, MT>(sp[2], e);
-    worker_batch<OPT, MASK, MT, GT, VEC, 0, 4>(a, sp, e, xb, ub, vb);
-    worker_batch<OPT, MASK, MT, GT, VEC, 4, MT - 4>(a, sp, e, xb, ub, vb);
+    worker_batch<OPT, MASK, MT, GT, VEC, 0, 4>(a, sp, sscale, e, xb, ub, vb);
+    worker_batch<OPT, MASK, MT, GT, VEC, 4, MT - 4>(a, sp, sscale, e, xb, ub, vb);
 }
 
 // ---- one thread's tile: MT workers x UN positions of VEC elements ------------------------
@@ -286,10 +288,11 @@ __device__ __forceinline__ void process_tile_split(const StepArgs &a, char *cons
 // Position j covers elements e0 + j * pstride .. + VEC - 1; positions >= npos are skipped.
 template <int OPT, int MASK, int MT, typename GT, bool POST, int VEC, int UN, bool FULL>
 __device__ __forceinline__ void process_tile(const StepArgs &a, char *const (*sp)[MT],
-                                             long long e0, int pstride, int npos) {
+                                             const float *sscale, long long e0, int pstride,
+                                             int npos) {
 #if DESLOC_SPLIT_LARGE_M
     if constexpr (!POST && MT > 4 && UN == 1 && OPT != OPT_SGDM) {
-        if (FULL || npos > 0) process_tile_split<OPT, MASK, MT, GT, VEC>(a, sp, e0);
+        if (FULL || npos > 0) process_tile_split<OPT, MASK, MT, GT, VEC>(a, sp, sscale, e0);
         return;
     }
 #endif
@@ -316,7 +319,7 @@ __device__ __forceinline__ void process_tile(const StepArgs &a, char *const (*sp
                 float g[MT], x[MT], u[MT], v[MT];
 #pragma unroll
                 for (int m = 0; m < MT; ++m) {
-                    g[m] = G[j][m].a[c];
+                    g[m] = G[j][m].a[c] * sscale[m];
                     x[m] = X[j][m].a[c];
                     u[m] = U[j][m].a[c];
                     v[m] = (OPT != OPT_SGDM) ? V[j][m].a[c] : 0.f;
@@ -350,8 +353,8 @@ struct UnrollFor {
 // One chunk of `count` elements for all MT workers: 128-bit path (with a scalar tail) when
 // every pointer is aligned, scalar path otherwise.
 template <int OPT, int MASK, int MT, typename GT, bool POST>
-__device__ __forceinline__ void process_chunk(const StepArgs &a, char *const (*sp)[MT], int count,
-                                              bool scalar_path) {
+__device__ __forceinline__ void process_chunk(const StepArgs &a, char *const (*sp)[MT],
+                                              const float *sscale, int count, bool scalar_path) {
     constexpr int UN = UnrollFor<MT>::value;
     const int tid = threadIdx.x;
     if (!scalar_path) {
@@ -360,23 +363,23 @@ __device__ __forceinline__ void process_chunk(const StepArgs &a, char *const (*s
 #pragma unroll 1
             for (int r = 0; r < 4 / UN; ++r)
                 process_tile<OPT, MASK, MT, GT, POST, 4, UN, true>(
-                    a, sp, static_cast<long long>(r * UN * BLOCK_THREADS + tid) * 4,
+                    a, sp, sscale, static_cast<long long>(r * UN * BLOCK_THREADS + tid) * 4,
                     BLOCK_THREADS * 4, UN);
         } else {
             const int n4 = count >> 2;
             for (int p0 = tid; p0 < n4; p0 += UN * BLOCK_THREADS) {
                 const int left = (n4 - p0 + BLOCK_THREADS - 1) / BLOCK_THREADS;
                 process_tile<OPT, MASK, MT, GT, POST, 4, UN, false>(
-                    a, sp, static_cast<long long>(p0) * 4, BLOCK_THREADS * 4,
+                    a, sp, sscale, static_cast<long long>(p0) * 4, BLOCK_THREADS * 4,
                     left < UN ? left : UN);
             }
             const int rem = count & 3;
             if (tid < rem)
-                process_tile<OPT, MASK, MT, GT, POST, 1, 1, true>(a, sp, (n4 << 2) + tid, 0, 1);
+                process_tile<OPT, MASK, MT, GT, POST, 1, 1, true>(a, sp, sscale, (n4 << 2) + tid, 0, 1);
         }
     } else {
         for (int e = tid; e < count; e += BLOCK_THREADS)
-            process_tile<OPT, MASK, MT, GT, POST, 1, 1, true>(a, sp, e, 0, 1);
+            process_tile<OPT, MASK, MT, GT, POST, 1, 1, true>(a, sp, sscale, e, 0, 1);
     }
 }
 
@@ -384,7 +387,9 @@ template <int OPT, int MASK, int MT, typename GT, bool POST>
 __global__ void __launch_bounds__(BLOCK_THREADS, (MT <= 4 ? 3 : ((OPT == OPT_SGDM || POST) ? 2 : DESLOC_MINB_LARGE_M)))
 desloc_step_kernel(const __grid_constant__ StepArgs a) {
     __shared__ char *sp[4][MT];
+    __shared__ float sscale[MT];
     const int tid = threadIdx.x;
+    if (tid < MT) sscale[tid] = a.gscale ? a.gscale[tid] : 1.f;  // published by the barriers below
     for (long long c = blockIdx.x; c < a.nchunks; c += gridDim.x) {
         constexpr int m0 = 0;
         const Chunk ch = a.chunks[c];
@@ -405,7 +410,7 @@ desloc_step_kernel(const __grid_constant__ StepArgs a) {
             misaligned = (reinterpret_cast<uintptr_t>(p) & need) != 0;
         }
         const int scalar_path = __syncthreads_or(misaligned);
-        process_chunk<OPT, MASK, MT, GT, POST>(a, sp, ch.count, scalar_path != 0);
+        process_chunk<OPT, MASK, MT, GT, POST>(a, sp, sscale, ch.count, scalar_path != 0);
     }
 }
 
@@ -421,6 +426,7 @@ desloc_local_kernel(const __grid_constant__ StepArgs a) {
     constexpr int SL = LOCAL_SLOTS;
     __shared__ char *sp[4][SL];
     __shared__ int scount[SL];
+    __shared__ float sscale[SL];  // all slots belong to one worker
     const int tid = threadIdx.x;
     const long long ngroups = (a.nchunks + SL - 1) / SL;
     const long long nitems = ngroups * a.M;
@@ -446,7 +452,10 @@ desloc_local_kernel(const __grid_constant__ StepArgs a) {
                         ch.start * static_cast<long long>(sizeof(GT));
             }
             sp[arr][sl] = p;
-            if (arr == 0) scount[sl] = cnt;
+            if (arr == 0) {
+                scount[sl] = cnt;
+                sscale[sl] = a.gscale ? a.gscale[m0] : 1.f;
+            }
             const unsigned need = (arr == 3 && sizeof(GT) == 2) ? 7u : 15u;
             slow = cnt != CHUNK_ELEMS || (reinterpret_cast<uintptr_t>(p) & need) != 0;
         }
@@ -454,7 +463,8 @@ desloc_local_kernel(const __grid_constant__ StepArgs a) {
 #pragma unroll 1
             for (int r = 0; r < 4; ++r)
                 process_tile<OPT, 0, SL, GT, false, 4, 1, true>(
-                    a, sp, static_cast<long long>(r * BLOCK_THREADS + tid) * 4, BLOCK_THREADS * 4, 1);
+                    a, sp, sscale, static_cast<long long>(r * BLOCK_THREADS + tid) * 4,
+                    BLOCK_THREADS * 4, 1);
         } else {
             // ragged group (a tensor's last chunk, an unaligned tensor, the list's end): slot by slot
 #pragma unroll 1
@@ -467,7 +477,7 @@ desloc_local_kernel(const __grid_constant__ StepArgs a) {
                                           reinterpret_cast<uintptr_t>(one[2][0]);
                 const bool mis = (bits & 15u) != 0 ||
                                  (reinterpret_cast<uintptr_t>(one[3][0]) & (sizeof(GT) == 2 ? 7u : 15u)) != 0;
-                process_chunk<OPT, 0, 1, GT, false>(a, one, cnt, mis);
+                process_chunk<OPT, 0, 1, GT, false>(a, one, sscale + sl, cnt, mis);
             }
         }
     }

@@ -1,0 +1,200 @@
+// Reductions around the DES-LOC step: per-worker gradient norms for norm-based clipping (the
+// clipping the paper's language-model runs used) and the relative rate of change of a state,
+// ||s_now - s_then||_2 / ||s_then||_2 (Section 5.1, "Metrics").
+//
+// Both are two-stage and deterministic: stage 1 writes one fp32 partial per (worker, chunk)
+// -- per-thread sums of up to 16 squares, a shuffle tree, then the eight warp sums in order;
+// stage 2 adds the partials of a worker in fp64 in a fixed pattern.  No atomics.
+#include "desloc_norms.cuh"
+
+namespace desloc {
+
+namespace {
+
+__device__ __forceinline__ float block_sum(float v, float *warp_sums) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_down_sync(0xffffffffu, v, off);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __syncthreads();  // warp_sums may still be read from the previous use
+    if (lane == 0) warp_sums[warp] = v;
+    __syncthreads();
+    float t = 0.f;
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 0; w < BLOCK_THREADS / 32; ++w) t += warp_sums[w];
+    }
+    return t;  // valid in thread 0
+}
+
+// partial[m * nchunks + c] = sum over chunk c of g^m squared.  Work item = (worker, chunk).
+template <typename GT>
+__global__ void __launch_bounds__(BLOCK_THREADS, 6)
+sumsq_kernel(const Chunk *chunks, long long nchunks, const void *const *g, int nt, int M,
+             float *partial) {
+    __shared__ float warp_sums[BLOCK_THREADS / 32];
+    const long long nitems = nchunks * M;
+    const int tid = threadIdx.x;
+    for (long long item = blockIdx.x; item < nitems; item += gridDim.x) {
+        const long long c = item % nchunks;
+        const int m = static_cast<int>(item / nchunks);
+        const Chunk ch = chunks[c];
+        const char *base = reinterpret_cast<const char *>(g[static_cast<long long>(m) * nt + ch.tensor]) +
+                           ch.start * static_cast<long long>(sizeof(GT));
+        const bool aligned = (reinterpret_cast<uintptr_t>(base) & (sizeof(GT) == 2 ? 7u : 15u)) == 0;
+        float acc = 0.f;
+        if (aligned) {
+            const int n4 = ch.count >> 2;
+            FV<4> v[4];
+            // up to four independent 128/64-bit loads per thread before the first use
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int p = tid + j * BLOCK_THREADS;
+                if (p < n4) v[j] = ld_grad<4, GT>(base, static_cast<long long>(p) * 4);
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int p = tid + j * BLOCK_THREADS;
+                if (p < n4) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) acc = fmaf(v[j].a[k], v[j].a[k], acc);
+                }
+            }
+            const int rem = ch.count & 3;
+            if (tid < rem) {
+                const float t = ld_grad<1, GT>(base, (n4 << 2) + tid).a[0];
+                acc = fmaf(t, t, acc);
+            }
+        } else {
+            for (int e = tid; e < ch.count; e += BLOCK_THREADS) {
+                const float t = ld_grad<1, GT>(base, e).a[0];
+                acc = fmaf(t, t, acc);
+            }
+        }
+        const float total = block_sum(acc, warp_sums);
+        if (tid == 0) partial[static_cast<long long>(m) * nchunks + c] = total;
+    }
+}
+
+// partial[(0|1) * M * nchunks + m * nchunks + c]: sum of (now - then)^2 and of then^2.
+__global__ void __launch_bounds__(BLOCK_THREADS, 6)
+relchange_kernel(const Chunk *chunks, long long nchunks, const float *const *now,
+                 const float *const *then, int nt, int M, float *partial) {
+    __shared__ float warp_sums[BLOCK_THREADS / 32];
+    const long long nitems = nchunks * M;
+    const int tid = threadIdx.x;
+    for (long long item = blockIdx.x; item < nitems; item += gridDim.x) {
+        const long long c = item % nchunks;
+        const int m = static_cast<int>(item / nchunks);
+        const Chunk ch = chunks[c];
+        const long long idx = static_cast<long long>(m) * nt + ch.tensor;
+        const char *pa = reinterpret_cast<const char *>(now[idx]) + ch.start * 4;
+        const char *pb = reinterpret_cast<const char *>(then[idx]) + ch.start * 4;
+        const bool aligned = ((reinterpret_cast<uintptr_t>(pa) | reinterpret_cast<uintptr_t>(pb)) & 15u) == 0;
+        float num = 0.f, den = 0.f;
+        if (aligned) {
+            const int n4 = ch.count >> 2;
+            for (int p = tid; p < n4; p += BLOCK_THREADS) {
+                const FV<4> a = ld_f32<4>(pa, static_cast<long long>(p) * 4);
+                const FV<4> b = ld_f32<4>(pb, static_cast<long long>(p) * 4);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const float d = a.a[k] - b.a[k];
+                    num = fmaf(d, d, num);
+                    den = fmaf(b.a[k], b.a[k], den);
+                }
+            }
+            const int rem = ch.count & 3;
+            if (tid < rem) {
+                const float a = ld_f32<1>(pa, (n4 << 2) + tid).a[0], b = ld_f32<1>(pb, (n4 << 2) + tid).a[0];
+                num = fmaf(a - b, a - b, num);
+                den = fmaf(b, b, den);
+            }
+        } else {
+            for (int e = tid; e < ch.count; e += BLOCK_THREADS) {
+                const float a = ld_f32<1>(pa, e).a[0], b = ld_f32<1>(pb, e).a[0];
+                num = fmaf(a - b, a - b, num);
+                den = fmaf(b, b, den);
+            }
+        }
+        const float tn = block_sum(num, warp_sums);
+        const float td = block_sum(den, warp_sums);
+        if (tid == 0) {
+            partial[static_cast<long long>(m) * nchunks + c] = tn;
+            partial[(static_cast<long long>(M) + m) * nchunks + c] = td;
+        }
+    }
+}
+
+// One block per row: out_sum[row] = sum of partial[row * n .. +n) in fp64, fixed pattern
+// (thread i adds entries i, i+256, ... in order; then a shared-memory tree).
+__device__ __forceinline__ double row_sum_f64(const float *row, long long n, double *sh) {
+    double acc = 0.0;
+    for (long long i = threadIdx.x; i < n; i += BLOCK_THREADS) acc += static_cast<double>(row[i]);
+    sh[threadIdx.x] = acc;
+    __syncthreads();
+    for (int s = BLOCK_THREADS / 2; s > 0; s >>= 1) {
+        if (threadIdx.x < s) sh[threadIdx.x] += sh[threadIdx.x + s];
+        __syncthreads();
+    }
+    const double r = sh[0];
+    __syncthreads();
+    return r;
+}
+
+// norms[m] = ||g^m||_2, scales[m] = min(1, max_norm / norms[m]) (1 when max_norm <= 0).
+__global__ void __launch_bounds__(BLOCK_THREADS)
+norm_finalize_kernel(const float *partial, long long nchunks, float max_norm, float *norms,
+                     float *scales) {
+    __shared__ double sh[BLOCK_THREADS];
+    const int m = blockIdx.x;
+    const double ss = row_sum_f64(partial + static_cast<long long>(m) * nchunks, nchunks, sh);
+    if (threadIdx.x == 0) {
+        const double nrm = sqrt(ss);
+        norms[m] = static_cast<float>(nrm);
+        scales[m] = (max_norm > 0.f && nrm > static_cast<double>(max_norm))
+                        ? static_cast<float>(static_cast<double>(max_norm) / nrm)
+                        : 1.f;
+    }
+}
+
+__global__ void __launch_bounds__(BLOCK_THREADS)
+relchange_finalize_kernel(const float *partial, long long nchunks, int M, float *out) {
+    __shared__ double sh[BLOCK_THREADS];
+    const int m = blockIdx.x;
+    const double num = row_sum_f64(partial + static_cast<long long>(m) * nchunks, nchunks, sh);
+    const double den = row_sum_f64(partial + (static_cast<long long>(M) + m) * nchunks, nchunks, sh);
+    if (threadIdx.x == 0) out[m] = static_cast<float>(sqrt(num) / sqrt(den));
+}
+
+unsigned grid_for(long long nitems) {
+    return static_cast<unsigned>(nitems < 0x7fffffffLL ? (nitems > 0 ? nitems : 1) : 0x7fffffffLL);
+}
+
+}  // namespace
+
+cudaError_t launch_grad_norms(const Chunk *chunks, long long nchunks, const void *const *g, int nt,
+                              int M, bool bf16, float max_norm, float *partial, float *norms,
+                              float *scales, cudaStream_t stream) {
+    const unsigned grid = grid_for(nchunks * M);
+    if (bf16)
+        sumsq_kernel<bf16_t><<<grid, BLOCK_THREADS, 0, stream>>>(chunks, nchunks, g, nt, M, partial);
+    else
+        sumsq_kernel<float><<<grid, BLOCK_THREADS, 0, stream>>>(chunks, nchunks, g, nt, M, partial);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    norm_finalize_kernel<<<M, BLOCK_THREADS, 0, stream>>>(partial, nchunks, max_norm, norms, scales);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_rel_change(const Chunk *chunks, long long nchunks, const float *const *now,
+                              const float *const *then, int nt, int M, float *partial, float *out,
+                              cudaStream_t stream) {
+    relchange_kernel<<<grid_for(nchunks * M), BLOCK_THREADS, 0, stream>>>(chunks, nchunks, now, then,
+                                                                          nt, M, partial);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    relchange_finalize_kernel<<<M, BLOCK_THREADS, 0, stream>>>(partial, nchunks, M, out);
+    return cudaGetLastError();
+}
+
+}  // namespace desloc

@@ -1,0 +1,18 @@
+// Launchers of the reduction kernels (gradient norms, relative state change).
+#pragma once
+#include "desloc_kernels.cuh"
+
+namespace desloc {
+
+// partial: scratch of at least M * nchunks floats; norms, scales: [M] floats, all on the device.
+// scales[m] = min(1, max_norm / ||g^m||_2), or 1 when max_norm <= 0.  Two launches.
+cudaError_t launch_grad_norms(const Chunk *chunks, long long nchunks, const void *const *g, int nt,
+                              int M, bool bf16, float max_norm, float *partial, float *norms,
+                              float *scales, cudaStream_t stream);
+
+// partial: scratch of at least 2 * M * nchunks floats; out[m] = ||now - then|| / ||then||.
+cudaError_t launch_rel_change(const Chunk *chunks, long long nchunks, const float *const *now,
+                              const float *const *then, int nt, int M, float *partial, float *out,
+                              cudaStream_t stream);
+
+}  // namespace desloc

@@ -151,6 +151,7 @@ extern "C" DESLOC_API int desloc_step_static(const desloc_config *cfg, float *co
         a.u = reinterpret_cast<float *const *>(tab + kMaxPointers);
         a.v = reinterpret_cast<float *const *>(tab + 2 * kMaxPointers);
         a.g = reinterpret_cast<const void *const *>(tab + 3 * kMaxPointers);
+        a.gscale = nullptr;
         a.nt = cfg->num_tensors;
         a.M = cfg->M;
         a.b1 = cfg->beta1;

@@ -64,6 +64,28 @@ class DesLoc:
         stream = torch.cuda.current_stream(self.device).cuda_stream
         return B.desloc_step(self.ctx, t, lr, clip_bound, self._grad_array(grads), stream)
 
+    def step_normclip(self, t: int, lr: float, grads, max_norm: float, clip_bound: float = 0.0) -> int:
+        """Step t with norm-based gradient clipping (per worker, over the whole tensor list)."""
+        stream = torch.cuda.current_stream(self.device).cuda_stream
+        return B.desloc_step_normclip(self.ctx, t, lr, clip_bound, max_norm,
+                                      self._grad_array(grads), stream)
+
+    def grad_norms(self):
+        """(norms, clip factors) of the latest step_normclip; synchronises the current stream."""
+        stream = torch.cuda.current_stream(self.device).cuda_stream
+        return B.desloc_get_grad_norms(self.ctx, self.M, stream)
+
+    def rel_change(self, array: int, then: Sequence[Sequence[torch.Tensor]]):
+        """Per-worker ||s - then|| / ||then|| against a snapshot (lists like x); synchronises."""
+        ptrs = []
+        for lst in then:
+            for t, n in zip(lst, self.numel):
+                if t.dtype != torch.float32 or t.numel() != n or not t.is_contiguous():
+                    raise ValueError("snapshot tensor of wrong dtype, size or layout")
+                ptrs.append(t.data_ptr())
+        stream = torch.cuda.current_stream(self.device).cuda_stream
+        return B.desloc_rel_change(self.ctx, array, ptrs, self.M, stream)
+
     def step_masked(self, mask: int, lr: float, grads, clip_bound: float = 0.0) -> None:
         stream = torch.cuda.current_stream(self.device).cuda_stream
         B.desloc_step_masked(self.ctx, mask, lr, clip_bound, self._grad_array(grads), stream)
