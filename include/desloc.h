@@ -170,6 +170,24 @@ DESLOC_API int desloc_get_grad_norms(desloc_ctx *ctx, float *norms_out, float *s
 DESLOC_API int desloc_rel_change(desloc_ctx *ctx, int32_t array, const float *const *then,
                                  float *out, void *stream);
 
+/*
+ * Change the set of workers between steps: add workers that start from the synchronised
+ * state, or drop some (the paper's robustness claim: because every state is eventually
+ * averaged, workers can join or leave; its experiment doubles the worker count mid-run,
+ * Section 6, RQ3).
+ *   M_new     : new worker count, 1..DESLOC_MAX_M.
+ *   x, u, v   : host arrays of M_new*num_tensors DEVICE pointers, indexed as in desloc_create().
+ *   first_new : workers 0..first_new-1 are taken as they are (normally the buffers of the
+ *               workers that stay; their contents are not touched).  Workers first_new..M_new-1
+ *               are new: every element of their x, u, v is overwritten with the mean over ALL
+ *               workers the context held before the call (fp64 sum in worker order).
+ *               first_new = M_new adds nobody (pure removal / re-ordering).
+ * This call allocates (the pointer tables are re-made for the new count), waits for `stream`
+ * before and after, and resets nothing else: counters and the step count continue.
+ */
+DESLOC_API int desloc_set_workers(desloc_ctx *ctx, int32_t M_new, int32_t first_new,
+                                  float *const *x, float *const *u, float *const *v, void *stream);
+
 /* Release the context and everything it allocated.  The caller's tensors are untouched.
    NULL is a no-op returning DESLOC_OK. */
 DESLOC_API int desloc_destroy(desloc_ctx *ctx);

@@ -74,6 +74,9 @@ def lib() -> ctypes.CDLL:
         L.desloc_oracle_norm_scales.argtypes = [ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
                                                 ctypes.c_void_p, ctypes.c_double, ctypes.c_void_p,
                                                 ctypes.c_void_p]
+        L.desloc_oracle_worker_mean.restype = None
+        L.desloc_oracle_worker_mean.argtypes = [ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
+                                                ctypes.c_void_p, ctypes.c_void_p]
         L.desloc_oracle_rel_change.restype = None
         L.desloc_oracle_rel_change.argtypes = [ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
                                                ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
@@ -116,6 +119,15 @@ def norm_scales(g, max_norm: float):
     lib().desloc_oracle_norm_scales(M, g.shape[1], g.shape[1], pg, float(max_norm),
                                     norms.ctypes.data, scales.ctypes.data)
     return norms, scales
+
+
+def worker_mean(s):
+    """E_m[s^m]: the fp32-rounded mean over workers of a float32 array of shape [M, n]."""
+    M = s.shape[0]
+    ps = _check(s, M, "s")
+    out = np.zeros(s.shape[1], dtype=np.float32)
+    lib().desloc_oracle_worker_mean(M, s.shape[1], s.shape[1], ps, out.ctypes.data)
+    return out
 
 
 def rel_change(now, then):

@@ -228,6 +228,15 @@ void desloc_oracle_norm_scales(int32_t M, int64_t n, int64_t stride, const float
 }
 
 /*
+ * Adding workers (Section 6, RQ3: the worker count is doubled mid-run; new workers start from
+ * the synchronised state): out[i] = E_m[s^m_i] over the M current workers, fp64 sum in the
+ * order m = 0..M-1, rounded to fp32 once.  The caller copies `out` into each new replica.
+ */
+void desloc_oracle_worker_mean(int32_t M, int64_t n, int64_t stride, const float *s, float *out) {
+    for (int64_t i = 0; i < n; ++i) out[i] = (float)worker_mean(s, stride, i, M);
+}
+
+/*
  * Relative change of a state over an interval, ||s_now - s_then||_2 / ||s_then||_2 per worker
  * (the rate-of-change measure of Section 5.1, "Metrics").
  */

@@ -78,6 +78,8 @@ _lib.desloc_step_masked.restype = ctypes.c_int
 _lib.desloc_step_masked.argtypes = [_P, ctypes.c_uint32, ctypes.c_float, ctypes.c_float, _PP, _P]
 _lib.desloc_destroy.restype = ctypes.c_int
 _lib.desloc_destroy.argtypes = [_P]
+_lib.desloc_set_workers.restype = ctypes.c_int
+_lib.desloc_set_workers.argtypes = [_P, ctypes.c_int32, ctypes.c_int32, _PP, _PP, _PP, _P]
 _lib.desloc_step_normclip.restype = ctypes.c_int
 _lib.desloc_step_normclip.argtypes = [_P, ctypes.c_int64, ctypes.c_float, ctypes.c_float,
                                       ctypes.c_float, _PP, _P, ctypes.POINTER(ctypes.c_uint32)]
@@ -217,6 +219,14 @@ def desloc_rel_change(ctx: int, array: int, then: Sequence[int], M: int, stream:
     if rc != DESLOC_OK:
         raise DeslocError(rc, "desloc_rel_change", _lib.desloc_last_cuda_error(ctx))
     return list(out)
+
+
+def desloc_set_workers(ctx: int, M_new: int, first_new: int, x, u, v, stream: int = 0) -> None:
+    """Replace the worker set; workers first_new.. are filled with the mean of the old workers."""
+    rc = _lib.desloc_set_workers(ctx, int(M_new), int(first_new), _ptr_array(x), _ptr_array(u),
+                                 _ptr_array(v), stream or None)
+    if rc != DESLOC_OK:
+        raise DeslocError(rc, "desloc_set_workers", _lib.desloc_last_cuda_error(ctx))
 
 
 def desloc_destroy(ctx: Optional[int]) -> None:

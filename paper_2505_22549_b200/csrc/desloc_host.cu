@@ -47,6 +47,59 @@ struct Slot {
     bool in_flight = false;
 };
 
+// Everything whose size depends on the worker count M (re-made by desloc_set_workers).
+struct WorkerRes {
+    void **d_tables = nullptr;  // [3][nptr] x, u, v
+    Slot slots[kSlots];
+    float *d_partial = nullptr;  // reductions: partial sums [2][M][nchunks]
+    float *d_norms = nullptr;    // [3][M]: gradient norms, clip factors, relative change
+    void **h_snap = nullptr;     // pinned pointer table for desloc_rel_change
+    void **d_snap = nullptr;
+};
+
+void free_worker_res(WorkerRes &r) {
+    for (Slot &s : r.slots) {
+        if (s.done) cudaEventDestroy(s.done);
+        if (s.host) cudaFreeHost(s.host);
+        if (s.dev) cudaFree(s.dev);
+        s = Slot();
+    }
+    if (r.d_tables) cudaFree(r.d_tables);
+    if (r.d_partial) cudaFree(r.d_partial);
+    if (r.d_norms) cudaFree(r.d_norms);
+    if (r.h_snap) cudaFreeHost(r.h_snap);
+    if (r.d_snap) cudaFree(r.d_snap);
+    r = WorkerRes();
+}
+
+// Allocates and fills the M-dependent resources; the device must be current.
+cudaError_t make_worker_res(WorkerRes &r, int M, int num_tensors, int64_t nchunks, bool has_v,
+                            float *const *x, float *const *u, float *const *v) {
+    const int64_t nptr = static_cast<int64_t>(M) * num_tensors;
+    std::vector<void *> tables(static_cast<size_t>(3 * nptr), nullptr);
+    for (int64_t i = 0; i < nptr; ++i) {
+        tables[i] = x[i];
+        tables[nptr + i] = u[i];
+        tables[2 * nptr + i] = has_v ? static_cast<void *>(v[i]) : nullptr;
+    }
+    cudaError_t e = cudaMalloc(&r.d_tables, tables.size() * sizeof(void *));
+    if (e == cudaSuccess)
+        e = cudaMemcpy(r.d_tables, tables.data(), tables.size() * sizeof(void *), cudaMemcpyHostToDevice);
+    const size_t npart = static_cast<size_t>(2) * M * static_cast<size_t>(nchunks);
+    if (e == cudaSuccess) e = cudaMalloc(&r.d_partial, npart * sizeof(float));
+    if (e == cudaSuccess) e = cudaMalloc(&r.d_norms, static_cast<size_t>(3) * M * sizeof(float));
+    if (e == cudaSuccess) e = cudaMemset(r.d_norms, 0, static_cast<size_t>(3) * M * sizeof(float));
+    if (e == cudaSuccess) e = cudaMallocHost(&r.h_snap, static_cast<size_t>(nptr) * sizeof(void *));
+    if (e == cudaSuccess) e = cudaMalloc(&r.d_snap, static_cast<size_t>(nptr) * sizeof(void *));
+    for (int i = 0; i < kSlots && e == cudaSuccess; ++i) {
+        Slot &s = r.slots[i];
+        e = cudaMallocHost(&s.host, static_cast<size_t>(nptr) * sizeof(void *));
+        if (e == cudaSuccess) e = cudaMalloc(&s.dev, static_cast<size_t>(nptr) * sizeof(void *));
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming);
+    }
+    return e;
+}
+
 }  // namespace
 
 struct desloc_ctx {
@@ -58,8 +111,7 @@ struct desloc_ctx {
     int64_t nptr = 0;  // M * num_tensors
     desloc::Chunk *d_chunks = nullptr;
     int64_t nchunks = 0;
-    void **d_tables = nullptr;  // [3][nptr] x, u, v
-    Slot slots[kSlots];
+    WorkerRes res;
     int next_slot = 0;
     int cur_slot = -1;           // slot holding the table equal to last_grads
     std::vector<const void *> last_grads;
@@ -68,11 +120,6 @@ struct desloc_ctx {
     int64_t launches = 0;
     int last_cuda_error = 0;
     int ctas_per_sm = 0;  // 0: one block per work item; > 0: persistent grid of that many per SM
-    // reductions: partial sums [2][M][nchunks], per-worker norms / clip factors / rel. change
-    float *d_partial = nullptr;
-    float *d_norms = nullptr;   // [3][M]: norms, scales, relative change
-    void **h_snap = nullptr;    // pinned pointer table for desloc_rel_change
-    void **d_snap = nullptr;
 };
 
 namespace {
@@ -117,17 +164,8 @@ uint32_t mask_at(const desloc_config *c, int64_t t) {
 
 void free_ctx(desloc_ctx *ctx) {
     if (!ctx) return;
-    for (Slot &s : ctx->slots) {
-        if (s.done) cudaEventDestroy(s.done);
-        if (s.host) cudaFreeHost(s.host);
-        if (s.dev) cudaFree(s.dev);
-    }
-    if (ctx->d_partial) cudaFree(ctx->d_partial);
-    if (ctx->d_norms) cudaFree(ctx->d_norms);
-    if (ctx->h_snap) cudaFreeHost(ctx->h_snap);
-    if (ctx->d_snap) cudaFree(ctx->d_snap);
+    free_worker_res(ctx->res);
     if (ctx->d_chunks) cudaFree(ctx->d_chunks);
-    if (ctx->d_tables) cudaFree(ctx->d_tables);
     delete ctx;
 }
 
@@ -136,10 +174,10 @@ int stage_grads(desloc_ctx *ctx, const void *const *grads, cudaStream_t stream, 
     const size_t bytes = static_cast<size_t>(ctx->nptr) * sizeof(void *);
     if (ctx->cur_slot >= 0 && stream == ctx->last_stream &&
         std::memcmp(ctx->last_grads.data(), grads, bytes) == 0) {
-        *dev_out = ctx->slots[ctx->cur_slot].dev;  // same pointers as last step: table is resident
+        *dev_out = ctx->res.slots[ctx->cur_slot].dev;  // same pointers as last step: table is resident
         return DESLOC_OK;
     }
-    Slot &s = ctx->slots[ctx->next_slot];
+    Slot &s = ctx->res.slots[ctx->next_slot];
     if (s.in_flight) {
         // Re-use of a slot whose kernel was enqueued kSlots table changes ago: wait for it.
         cudaError_t e = cudaEventSynchronize(s.done);
@@ -185,13 +223,13 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
             e = desloc::launch_grad_norms(ctx->d_chunks, ctx->nchunks,
                                           reinterpret_cast<const void *const *>(d_g), c.num_tensors,
                                           c.M, c.grad_dtype == DESLOC_BF16, max_norm,
-                                          ctx->d_partial, ctx->d_norms, ctx->d_norms + c.M, stream);
+                                          ctx->res.d_partial, ctx->res.d_norms, ctx->res.d_norms + c.M, stream);
             if (e != cudaSuccess) {
                 rc = cuda_fail(ctx, e);
                 break;
             }
             ctx->launches += 2;
-            d_gscale = ctx->d_norms + c.M;
+            d_gscale = ctx->res.d_norms + c.M;
         }
 
         // The mean of one replica is the replica: M = 1 always runs the local kernel.
@@ -210,9 +248,9 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
         desloc::StepArgs a{};
         a.chunks = ctx->d_chunks;
         a.nchunks = ctx->nchunks;
-        a.x = reinterpret_cast<float *const *>(ctx->d_tables);
-        a.u = reinterpret_cast<float *const *>(ctx->d_tables + ctx->nptr);
-        a.v = reinterpret_cast<float *const *>(ctx->d_tables + 2 * ctx->nptr);
+        a.x = reinterpret_cast<float *const *>(ctx->res.d_tables);
+        a.u = reinterpret_cast<float *const *>(ctx->res.d_tables + ctx->nptr);
+        a.v = reinterpret_cast<float *const *>(ctx->res.d_tables + 2 * ctx->nptr);
         a.g = reinterpret_cast<const void *const *>(d_g);
         a.gscale = d_gscale;
         a.nt = c.num_tensors;
@@ -246,7 +284,7 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
             break;
         }
         ctx->launches += 1;
-        Slot &s = ctx->slots[ctx->cur_slot];
+        Slot &s = ctx->res.slots[ctx->cur_slot];
         e = cudaEventRecord(s.done, stream);
         if (e != cudaSuccess) {
             rc = cuda_fail(ctx, e);
@@ -317,7 +355,6 @@ int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *const *x, f
     desloc_ctx *ctx = new (std::nothrow) desloc_ctx();
     if (!ctx) return DESLOC_E_NOMEM;
     std::vector<desloc::Chunk> chunks;
-    std::vector<void *> tables;
     try {
         ctx->numel.assign(cfg->numel, cfg->numel + cfg->num_tensors);
         ctx->last_grads.assign(static_cast<size_t>(nptr), nullptr);
@@ -330,12 +367,6 @@ int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *const *x, f
                 ch.count = static_cast<int32_t>(left < desloc::CHUNK_ELEMS ? left : desloc::CHUNK_ELEMS);
                 chunks.push_back(ch);
             }
-        tables.resize(static_cast<size_t>(3 * nptr), nullptr);
-        for (int64_t i = 0; i < nptr; ++i) {
-            tables[i] = x[i];
-            tables[nptr + i] = u[i];
-            tables[2 * nptr + i] = v ? static_cast<void *>(v[i]) : nullptr;
-        }
     } catch (const std::bad_alloc &) {
         delete ctx;
         return DESLOC_E_NOMEM;
@@ -353,24 +384,16 @@ int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *const *x, f
     if (e == cudaSuccess)
         e = cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, cuda_device);
     if (e == cudaSuccess) e = cudaMalloc(&ctx->d_chunks, chunks.size() * sizeof(desloc::Chunk));
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_tables, tables.size() * sizeof(void *));
     if (e == cudaSuccess)
         e = cudaMemcpy(ctx->d_chunks, chunks.data(), chunks.size() * sizeof(desloc::Chunk),
                        cudaMemcpyHostToDevice);
-    if (e == cudaSuccess)
-        e = cudaMemcpy(ctx->d_tables, tables.data(), tables.size() * sizeof(void *),
-                       cudaMemcpyHostToDevice);
-    const size_t npart = static_cast<size_t>(2) * cfg->M * chunks.size();
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_partial, npart * sizeof(float));
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_norms, static_cast<size_t>(3) * cfg->M * sizeof(float));
-    if (e == cudaSuccess) e = cudaMemset(ctx->d_norms, 0, static_cast<size_t>(3) * cfg->M * sizeof(float));
-    if (e == cudaSuccess) e = cudaMallocHost(&ctx->h_snap, static_cast<size_t>(nptr) * sizeof(void *));
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_snap, static_cast<size_t>(nptr) * sizeof(void *));
-    for (int i = 0; i < kSlots && e == cudaSuccess; ++i) {
-        Slot &s = ctx->slots[i];
-        e = cudaMallocHost(&s.host, static_cast<size_t>(nptr) * sizeof(void *));
-        if (e == cudaSuccess) e = cudaMalloc(&s.dev, static_cast<size_t>(nptr) * sizeof(void *));
-        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming);
+    if (e == cudaSuccess) {
+        try {
+            e = make_worker_res(ctx->res, cfg->M, cfg->num_tensors, ctx->nchunks,
+                                cfg->opt != DESLOC_SGDM, x, u, v);
+        } catch (const std::bad_alloc &) {
+            e = cudaErrorMemoryAllocation;
+        }
     }
     if (dev_before >= 0 && dev_before != cuda_device) cudaSetDevice(dev_before);
     if (e != cudaSuccess) {
@@ -417,9 +440,9 @@ int desloc_get_grad_norms(desloc_ctx *ctx, float *norms_out, float *scales_out, 
     const size_t bytes = static_cast<size_t>(ctx->cfg.M) * sizeof(float);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaSuccess;
-    if (norms_out) e = cudaMemcpyAsync(norms_out, ctx->d_norms, bytes, cudaMemcpyDeviceToHost, st);
+    if (norms_out) e = cudaMemcpyAsync(norms_out, ctx->res.d_norms, bytes, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess && scales_out)
-        e = cudaMemcpyAsync(scales_out, ctx->d_norms + ctx->cfg.M, bytes, cudaMemcpyDeviceToHost, st);
+        e = cudaMemcpyAsync(scales_out, ctx->res.d_norms + ctx->cfg.M, bytes, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     return e == cudaSuccess ? DESLOC_OK : cuda_fail(ctx, e);
 }
@@ -437,15 +460,15 @@ int desloc_rel_change(desloc_ctx *ctx, int32_t array, const float *const *then, 
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     const size_t tbytes = static_cast<size_t>(ctx->nptr) * sizeof(void *);
     // The call ends with a stream synchronisation, so the pinned table is free again on return.
-    std::memcpy(ctx->h_snap, then, tbytes);
-    e = cudaMemcpyAsync(ctx->d_snap, ctx->h_snap, tbytes, cudaMemcpyHostToDevice, st);
-    float *d_out = ctx->d_norms + 2 * ctx->cfg.M;
+    std::memcpy(ctx->res.h_snap, then, tbytes);
+    e = cudaMemcpyAsync(ctx->res.d_snap, ctx->res.h_snap, tbytes, cudaMemcpyHostToDevice, st);
+    float *d_out = ctx->res.d_norms + 2 * ctx->cfg.M;
     if (e == cudaSuccess)
         e = desloc::launch_rel_change(
             ctx->d_chunks, ctx->nchunks,
-            reinterpret_cast<const float *const *>(ctx->d_tables + array * ctx->nptr),
-            reinterpret_cast<const float *const *>(ctx->d_snap), ctx->cfg.num_tensors, ctx->cfg.M,
-            ctx->d_partial, d_out, st);
+            reinterpret_cast<const float *const *>(ctx->res.d_tables + array * ctx->nptr),
+            reinterpret_cast<const float *const *>(ctx->res.d_snap), ctx->cfg.num_tensors, ctx->cfg.M,
+            ctx->res.d_partial, d_out, st);
     if (e == cudaSuccess) {
         ctx->launches += 2;
         e = cudaMemcpyAsync(out, d_out, static_cast<size_t>(ctx->cfg.M) * sizeof(float),
@@ -454,6 +477,64 @@ int desloc_rel_change(desloc_ctx *ctx, int32_t array, const float *const *then, 
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (dev_before != ctx->device) cudaSetDevice(dev_before);
     return e == cudaSuccess ? DESLOC_OK : cuda_fail(ctx, e);
+}
+
+int desloc_set_workers(desloc_ctx *ctx, int32_t M_new, int32_t first_new, float *const *x,
+                       float *const *u, float *const *v, void *stream) {
+    if (!ctx || !x || !u) return DESLOC_E_NULL;
+    const bool has_v = ctx->cfg.opt != DESLOC_SGDM;
+    if (has_v && !v) return DESLOC_E_NULL;
+    if (M_new < 1 || M_new > DESLOC_MAX_M || first_new < 0 || first_new > M_new) return DESLOC_E_RANGE;
+    const int nt = ctx->cfg.num_tensors;
+    const int64_t nptr_new = static_cast<int64_t>(M_new) * nt;
+    for (int64_t i = 0; i < nptr_new; ++i) {
+        if (!x[i] || !u[i] || (has_v && !v[i])) return DESLOC_E_NULL;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int dev_before = -1;
+    cudaError_t e = cudaGetDevice(&dev_before);
+    if (e == cudaSuccess && dev_before != ctx->device) e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    // Earlier steps must have finished with the old tables before they are replaced.
+    e = cudaStreamSynchronize(st);
+    WorkerRes fresh;
+    if (e == cudaSuccess) {
+        try {
+            e = make_worker_res(fresh, M_new, nt, ctx->nchunks, has_v, x, u, v);
+            ctx->last_grads.assign(static_cast<size_t>(nptr_new), nullptr);
+        } catch (const std::bad_alloc &) {
+            e = cudaErrorMemoryAllocation;
+        }
+    }
+    const int n_new = M_new - first_new;
+    if (e == cudaSuccess && n_new > 0) {
+        // New replicas start from the mean of ALL replicas the context held so far.
+        const int n_arr = has_v ? 3 : 2;
+        for (int arr = 0; arr < n_arr && e == cudaSuccess; ++arr)
+            e = desloc::launch_mean_fill(
+                ctx->d_chunks, ctx->nchunks,
+                reinterpret_cast<const float *const *>(ctx->res.d_tables + arr * ctx->nptr), ctx->cfg.M,
+                reinterpret_cast<float *const *>(fresh.d_tables + arr * nptr_new +
+                                                 static_cast<int64_t>(first_new) * nt),
+                n_new, nt, st);
+        if (e == cudaSuccess) ctx->launches += n_arr;
+    }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    int rc = DESLOC_OK;
+    if (e == cudaSuccess) {
+        free_worker_res(ctx->res);
+        ctx->res = fresh;
+        ctx->cfg.M = M_new;
+        ctx->nptr = nptr_new;
+        ctx->next_slot = 0;
+        ctx->cur_slot = -1;
+    } else {
+        free_worker_res(fresh);
+        rc = (e == cudaErrorMemoryAllocation) ? DESLOC_E_NOMEM : cuda_fail(ctx, e);
+        (void)cudaGetLastError();
+    }
+    if (dev_before != ctx->device) cudaSetDevice(dev_before);
+    return rc;
 }
 
 int desloc_destroy(desloc_ctx *ctx) {

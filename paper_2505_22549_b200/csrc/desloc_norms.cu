@@ -166,6 +166,24 @@ relchange_finalize_kernel(const float *partial, long long nchunks, int M, float 
     if (threadIdx.x == 0) out[m] = static_cast<float>(sqrt(num) / sqrt(den));
 }
 
+// dst^j[i] = mean over the M_src source replicas of src^m[i] (fp64 sum in the order
+// m = 0..M_src-1, rounded once), for every destination replica j.  Work item = chunk.
+__global__ void __launch_bounds__(BLOCK_THREADS, 4)
+mean_fill_kernel(const Chunk *chunks, long long nchunks, const float *const *src, int m_src,
+                 float *const *dst, int m_dst, int nt) {
+    for (long long c = blockIdx.x; c < nchunks; c += gridDim.x) {
+        const Chunk ch = chunks[c];
+        for (int e = threadIdx.x; e < ch.count; e += BLOCK_THREADS) {
+            double acc = 0.0;
+            for (int m = 0; m < m_src; ++m)
+                acc += static_cast<double>(src[static_cast<long long>(m) * nt + ch.tensor][ch.start + e]);
+            const float mean = static_cast<float>(acc / static_cast<double>(m_src));
+            for (int j = 0; j < m_dst; ++j)
+                dst[static_cast<long long>(j) * nt + ch.tensor][ch.start + e] = mean;
+        }
+    }
+}
+
 unsigned grid_for(long long nitems) {
     return static_cast<unsigned>(nitems < 0x7fffffffLL ? (nitems > 0 ? nitems : 1) : 0x7fffffffLL);
 }
@@ -194,6 +212,13 @@ cudaError_t launch_rel_change(const Chunk *chunks, long long nchunks, const floa
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     relchange_finalize_kernel<<<M, BLOCK_THREADS, 0, stream>>>(partial, nchunks, M, out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_mean_fill(const Chunk *chunks, long long nchunks, const float *const *src,
+                             int m_src, float *const *dst, int m_dst, int nt, cudaStream_t stream) {
+    mean_fill_kernel<<<grid_for(nchunks), BLOCK_THREADS, 0, stream>>>(chunks, nchunks, src, m_src,
+                                                                      dst, m_dst, nt);
     return cudaGetLastError();
 }
 

@@ -15,4 +15,9 @@ cudaError_t launch_rel_change(const Chunk *chunks, long long nchunks, const floa
                               const float *const *then, int nt, int M, float *partial, float *out,
                               cudaStream_t stream);
 
+// Every element of the m_dst destination replicas := mean over the m_src source replicas.
+// src / dst are device tables indexed [m * nt + tensor].
+cudaError_t launch_mean_fill(const Chunk *chunks, long long nchunks, const float *const *src,
+                             int m_src, float *const *dst, int m_dst, int nt, cudaStream_t stream);
+
 }  // namespace desloc

@@ -86,6 +86,21 @@ class DesLoc:
         stream = torch.cuda.current_stream(self.device).cuda_stream
         return B.desloc_rel_change(self.ctx, array, ptrs, self.M, stream)
 
+    def set_workers(self, x, u, v, first_new: int) -> None:
+        """New worker set (lists like the constructor's); workers first_new.. start from the mean
+        of the current workers.  Synchronises the current stream."""
+        M = len(x)
+        for arrs in (x, u) + ((v,) if v is not None else ()):
+            if len(arrs) != M or any([int(t.numel()) for t in lst] != self.numel for lst in arrs):
+                raise ValueError("every worker needs the same tensor list")
+        flat = lambda a: [t.data_ptr() for lst in a for t in lst]
+        stream = torch.cuda.current_stream(self.device).cuda_stream
+        B.desloc_set_workers(self.ctx, M, first_new, flat(x), flat(u),
+                             flat(v) if v is not None else None, stream)
+        self._keep = (x, u, v)
+        self.M = M
+        self._gkey = self._garr = None
+
     def step_masked(self, mask: int, lr: float, grads, clip_bound: float = 0.0) -> None:
         stream = torch.cuda.current_stream(self.device).cuda_stream
         B.desloc_step_masked(self.ctx, mask, lr, clip_bound, self._grad_array(grads), stream)

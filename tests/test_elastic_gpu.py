@@ -1,0 +1,110 @@
+"""Workers joining and leaving between steps (the paper doubles the worker count mid-run):
+new replicas start from the mean of the current ones; the run continues and still matches the
+oracle doing the same thing on the host."""
+import numpy as np
+import pytest
+import torch
+
+import desloc_inputs as di
+import oracle
+from _util import State, compare_per_tensor, f32r, oracle_cfg
+from test_parity_gpu import make_engine
+
+pytestmark = pytest.mark.gpu
+
+
+def _host(bufs):
+    return np.ascontiguousarray(np.stack([b.float().cpu().numpy() for b in bufs]), dtype=np.float32)
+
+
+@pytest.mark.parametrize("name", ["cfg2_adam_135m", "cfg5_sgdm_desloc", "cfg3_adopt_360m"])
+def test_double_then_shrink_worker_count(name):
+    import paper_2505_22549_b200 as d
+    base = di.mini(di.WORKLOADS[name], T=18).replace(M=2, K=(2, 3, 4))
+    dev = torch.device("cuda:0")
+    st = State(base.replace(M=4), dev)          # room for four workers; two are used at first
+    w2 = base
+    x, u = st.x[:2], st.u[:2]
+    v = st.v[:2] if st.v is not None else None
+    eng = d.DesLoc(st.views(x), st.views(u), st.views(v) if v is not None else None, opt=w2.opt,
+                   grad_dtype=w2.grad_dtype, beta1=w2.beta1, beta2=w2.beta2, eps=w2.eps,
+                   weight_decay=w2.weight_decay, clip_rho=w2.clip_rho, K=w2.K,
+                   flags=d.DESLOC_FLAG_ADOPT_NORM_CLIP if w2.adopt_norm_clip else 0)
+    ox, ou = _host(x), _host(u)
+    ov = _host(v) if v is not None else None
+    M = 2
+    w4 = base.replace(M=4)
+
+    def step(t):
+        nonlocal ox, ou, ov
+        wl = w4 if M == 4 else (base.replace(M=M))
+        for m in range(M):
+            di.fill_grads_(w4, t, m, st.g[m], align=4)
+        lr, cb = f32r(base.lr), f32r(base.clip_bound(t))
+        mk = eng.step(t, lr, st.views(st.g[:M]), clip_bound=cb)
+        mo = oracle.step(oracle_cfg(wl), t, lr, ox, ou, ov, _host(st.g[:M]), clip_bound=cb)
+        assert mk == mo
+
+    for t in range(0, 6):
+        step(t)
+    # ---- double: workers 2, 3 join, initialised from the mean of workers 0, 1
+    torch.cuda.synchronize()
+    before = [_host(b[:2]) for b in (st.x, st.u) + ((st.v,) if st.v is not None else ())]
+    for bufs in (st.x, st.u) + ((st.v,) if st.v is not None else ()):
+        bufs[2].fill_(float("nan"))             # whatever was there must be overwritten
+        bufs[3].fill_(float("nan"))
+    eng.set_workers(st.views(st.x), st.views(st.u), st.views(st.v) if st.v is not None else None,
+                    first_new=2)
+    M = 4
+    grow = lambda a: np.ascontiguousarray(np.concatenate([a, np.tile(oracle.worker_mean(a), (2, 1))]))
+    ox, ou = grow(ox), grow(ou)
+    ov = grow(ov) if ov is not None else None
+    valid = st.valid_mask()
+    after = [_host(b) for b in (st.x, st.u) + ((st.v,) if st.v is not None else ())]
+    for b4, aft in zip(before, after):
+        want = oracle.worker_mean(b4)
+        assert np.array_equal(aft[:2], b4)                       # survivors untouched
+        for j in (2, 3):                                         # joiners = mean, bit for bit
+            assert np.array_equal(aft[j][valid], want[valid])
+    for t in range(6, 12):
+        step(t)
+    # ---- shrink: workers 1 and 3 leave; survivors keep their buffers
+    keep = [0, 2]
+    eng.set_workers(st.views([st.x[i] for i in keep]), st.views([st.u[i] for i in keep]),
+                    st.views([st.v[i] for i in keep]) if st.v is not None else None, first_new=2)
+    ox, ou = np.ascontiguousarray(ox[keep]), np.ascontiguousarray(ou[keep])
+    ov = np.ascontiguousarray(ov[keep]) if ov is not None else None
+    M = 2
+    gsel = [st.g[0], st.g[1]]
+    for t in range(12, 18):
+        for m in range(2):
+            di.fill_grads_(w4, t, m, gsel[m], align=4)
+        lr, cb = f32r(base.lr), f32r(base.clip_bound(t))
+        eng.step(t, lr, st.views(gsel), clip_bound=cb)
+        oracle.step(oracle_cfg(base), t, lr, ox, ou, ov, _host(gsel), clip_bound=cb)
+    torch.cuda.synchronize()
+    sub = State.__new__(State)
+    sub.offs, sub.w = st.offs, base
+    compare_per_tensor(sub, _host([st.x[i] for i in keep]), ox, "x")
+    compare_per_tensor(sub, _host([st.u[i] for i in keep]), ou, "u")
+    if ov is not None:
+        compare_per_tensor(sub, _host([st.v[i] for i in keep]), ov, "v")
+    assert eng.counters()[0] == 18
+    eng.close()
+
+
+def test_set_workers_rejects_bad_arguments():
+    import paper_2505_22549_b200 as d
+    dev = torch.device("cuda:0")
+    bufs = [torch.zeros(8, device=dev) for _ in range(6)]
+    cfg = d.make_config(2, [8], "adam", "f32")
+    p = [b.data_ptr() for b in bufs]
+    ctx = d.desloc_create(cfg, p[0:2], p[2:4], p[4:6], 0)
+    for M_new, first in [(0, 0), (65, 0), (2, 3), (2, -1)]:
+        with pytest.raises(d.DeslocError) as e:
+            d.desloc_set_workers(ctx, M_new, first, p[0:2], p[2:4], p[4:6])
+        assert e.value.status == d.DESLOC_E_RANGE
+    with pytest.raises(d.DeslocError) as e:
+        d.desloc_set_workers(ctx, 2, 2, [p[0], 0], p[2:4], p[4:6])
+    assert e.value.status == d.DESLOC_E_NULL
+    d.desloc_destroy(ctx)

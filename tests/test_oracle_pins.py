@@ -551,3 +551,19 @@ def test_rel_change_closed_forms():
     assert np.allclose(out, [1.0, 0.0])
     now2 = f32([[1.0, 2.0, 5.0], [0.0, 0.0, 0.0]])      # diff (0,0,3)/3 ; (3,0,4)/5
     assert np.allclose(oracle.rel_change(now2, then), [1.0, 1.0])
+
+
+# --------------------------------------------------------------------------- adding workers
+def test_worker_mean_closed_forms_and_doubling_keeps_the_mean():
+    s = f32([[1.0, -2.0, 0.5], [3.0, 2.0, 0.25], [2.0, 0.0, 0.0]])
+    assert np.array_equal(oracle.worker_mean(s), f32([2.0, 0.0, 0.25]))
+    # identical replicas: the mean is that replica, bit for bit, for any M
+    rng = np.random.default_rng(12)
+    row = rng.normal(size=33).astype(np.float32)
+    for M in (2, 3, 5, 8):
+        assert np.array_equal(oracle.worker_mean(f32(np.tile(row, (M, 1)))), row)
+    # new workers that start from the mean leave the worker-mean unchanged (exact on dyadics)
+    base = rng.integers(-8, 9, size=(4, 16)).astype(np.float32)
+    mean = oracle.worker_mean(f32(base))
+    doubled = f32(np.concatenate([base, np.tile(mean, (4, 1))]))
+    assert np.array_equal(oracle.worker_mean(doubled), mean)
