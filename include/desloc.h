@@ -128,6 +128,14 @@ DESLOC_API int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *
  *   mask_out     : if not NULL receives the sync mask that was applied.
  * Errors: a failed launch is returned by this call; an asynchronous execution error surfaces
  * in a later call or at the caller's next synchronisation.
+ *
+ * Stream capture (CUDA graphs, for small launch-bound problems): the call may be made while
+ * `stream` is capturing if either M*num_tensors <= 32 (the gradient pointers then travel in
+ * the kernel parameters) or `grads` holds the same pointers as the previous, un-captured call
+ * on that stream; otherwise it returns DESLOC_E_INVALID and captures nothing.  t, lr_t and
+ * clip_bound_t are frozen into the captured launch, so a replayed graph repeats the same mask
+ * sequence: capture a window of lcm(Kx, Ku, Kv) steps starting at a multiple of it.  Counters
+ * and the launch count advance when a call is captured, not when the graph is replayed.
  */
 DESLOC_API int desloc_step(desloc_ctx *ctx, int64_t t, float lr_t, float clip_bound_t,
                 const void *const *grads, void *stream, uint32_t *mask_out);

@@ -24,7 +24,7 @@ __device__ __forceinline__ Ptrs worker_ptrs(const StepArgs &a, const Chunk &ch, 
     p.x = reinterpret_cast<char *>(a.x[idx]) + ch.start * 4;
     p.u = reinterpret_cast<char *>(a.u[idx]) + ch.start * 4;
     p.v = (OPT != OPT_SGDM) ? reinterpret_cast<char *>(a.v[idx]) + ch.start * 4 : nullptr;
-    p.g = reinterpret_cast<const char *>(a.g[idx]) + ch.start * static_cast<long long>(sizeof(GT));
+    p.g = reinterpret_cast<const char *>(grad_ptr(a, idx)) + ch.start * static_cast<long long>(sizeof(GT));
     return p;
 }
 

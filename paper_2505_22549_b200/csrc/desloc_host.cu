@@ -214,9 +214,30 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
     }
     int rc = DESLOC_OK;
     do {
+        // Under stream capture nothing may be staged through the pinned ring (a replay would
+        // read whatever the ring holds by then) and no event of the ring may be recorded.
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        e = cudaStreamIsCapturing(stream, &cap);
+        if (e != cudaSuccess) {
+            rc = cuda_fail(ctx, e);
+            break;
+        }
+        const bool capturing = cap != cudaStreamCaptureStatusNone;
         void **d_g = nullptr;
-        rc = stage_grads(ctx, grads, stream, &d_g);
-        if (rc != DESLOC_OK) break;
+        bool inline_g = false;
+        if (!capturing) {
+            rc = stage_grads(ctx, grads, stream, &d_g);
+            if (rc != DESLOC_OK) break;
+        } else if (ctx->cur_slot >= 0 && stream == ctx->last_stream &&
+                   std::memcmp(ctx->last_grads.data(), grads,
+                               static_cast<size_t>(ctx->nptr) * sizeof(void *)) == 0) {
+            d_g = ctx->res.slots[ctx->cur_slot].dev;  // table already resident
+        } else if (ctx->nptr <= desloc::INLINE_PTRS && max_norm <= 0.f) {
+            inline_g = true;  // pointers travel in the kernel parameters
+        } else {
+            rc = DESLOC_E_INVALID;  // stage these pointers with one un-captured step first
+            break;
+        }
 
         const float *d_gscale = nullptr;
         if (max_norm > 0.f) {
@@ -252,6 +273,8 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
         a.u = reinterpret_cast<float *const *>(ctx->res.d_tables + ctx->nptr);
         a.v = reinterpret_cast<float *const *>(ctx->res.d_tables + 2 * ctx->nptr);
         a.g = reinterpret_cast<const void *const *>(d_g);
+        if (inline_g)
+            for (int64_t i = 0; i < ctx->nptr; ++i) a.g_inline[i] = grads[i];
         a.gscale = d_gscale;
         a.nt = c.num_tensors;
         a.M = c.M;
@@ -284,13 +307,15 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
             break;
         }
         ctx->launches += 1;
-        Slot &s = ctx->res.slots[ctx->cur_slot];
-        e = cudaEventRecord(s.done, stream);
-        if (e != cudaSuccess) {
-            rc = cuda_fail(ctx, e);
-            break;
+        if (!capturing) {
+            Slot &s = ctx->res.slots[ctx->cur_slot];
+            e = cudaEventRecord(s.done, stream);
+            if (e != cudaSuccess) {
+                rc = cuda_fail(ctx, e);
+                break;
+            }
+            s.in_flight = true;
         }
-        s.in_flight = true;
         ctx->counters[0] += 1;
         ctx->counters[1] += (mask & DESLOC_SYNC_X) ? 1 : 0;
         ctx->counters[2] += (mask & DESLOC_SYNC_U) ? 1 : 0;

@@ -42,13 +42,16 @@ struct __align__(16) Chunk {
     int64_t start;   // first element within the tensor
 };
 
+constexpr int INLINE_PTRS = 32;  // gradient pointers that fit in the kernel parameters
+
 struct StepArgs {
     const Chunk *chunks;
     long long nchunks;
     float *const *x;  // device tables [M * nt], entry m * nt + k
     float *const *u;
     float *const *v;
-    const void *const *g;
+    const void *const *g;                // device table, or nullptr: use g_inline
+    const void *g_inline[INLINE_PTRS];   // small problems under stream capture (no table upload)
     const float *gscale;  // per-worker factor applied to g before the clip, or nullptr (= 1)
     int nt;
     int M;
@@ -61,6 +64,10 @@ struct StepArgs {
     float rho;        // coordinate clip radius, +inf when off
     float cbound;     // ADOPT normalised-gradient bound, +inf when off
 };
+
+__device__ __forceinline__ const void *grad_ptr(const StepArgs &a, long long idx) {
+    return a.g ? a.g[idx] : a.g_inline[idx];
+}
 
 struct bf16_t {
     uint16_t bits;
@@ -403,7 +410,7 @@ desloc_step_kernel(const __grid_constant__ StepArgs a) {
             if (arr == 1) p = reinterpret_cast<char *>(a.u[idx]) + ch.start * 4;
             if (arr == 2 && OPT != OPT_SGDM) p = reinterpret_cast<char *>(a.v[idx]) + ch.start * 4;
             if (arr == 3)
-                p = const_cast<char *>(reinterpret_cast<const char *>(a.g[idx])) +
+                p = const_cast<char *>(reinterpret_cast<const char *>(grad_ptr(a, idx))) +
                     ch.start * static_cast<long long>(sizeof(GT));
             sp[arr][m] = p;
             const unsigned need = (arr == 3 && sizeof(GT) == 2) ? 7u : 15u;
@@ -448,7 +455,7 @@ desloc_local_kernel(const __grid_constant__ StepArgs a) {
                 if (arr == 1) p = reinterpret_cast<char *>(a.u[idx]) + ch.start * 4;
                 if (arr == 2 && OPT != OPT_SGDM) p = reinterpret_cast<char *>(a.v[idx]) + ch.start * 4;
                 if (arr == 3)
-                    p = const_cast<char *>(reinterpret_cast<const char *>(a.g[idx])) +
+                    p = const_cast<char *>(reinterpret_cast<const char *>(grad_ptr(a, idx))) +
                         ch.start * static_cast<long long>(sizeof(GT));
             }
             sp[arr][sl] = p;
