@@ -224,7 +224,8 @@ DESLOC_API int desloc_set_launch_shape(desloc_ctx *ctx, int32_t ctas_per_sm);
 DESLOC_API int64_t desloc_plan_chunks(const int64_t *numel, int32_t num_tensors, int64_t chunk_elems,
                            int64_t *out, int64_t cap);
 
-/* Elements per chunk used by contexts of this build. */
+/* Elements per chunk used by contexts of this build (problems of fewer than 296 such chunks
+   are cut into chunks a quarter of this size). */
 DESLOC_API int64_t desloc_chunk_elems(void);
 
 /*

@@ -380,16 +380,22 @@ int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *const *x, f
     desloc_ctx *ctx = new (std::nothrow) desloc_ctx();
     if (!ctx) return DESLOC_E_NOMEM;
     std::vector<desloc::Chunk> chunks;
+    // Small problems (fewer full-size chunks than two per SM of a B200) are latency-bound:
+    // quarter-size chunks spread them over four times as many blocks, one tile per thread.
+    int64_t full_chunks = 0;
+    for (int32_t k = 0; k < cfg->num_tensors; ++k)
+        full_chunks += (cfg->numel[k] + desloc::CHUNK_ELEMS - 1) / desloc::CHUNK_ELEMS;
+    const int64_t chunk_elems = full_chunks < 2 * 148 ? desloc::CHUNK_ELEMS / 4 : desloc::CHUNK_ELEMS;
     try {
         ctx->numel.assign(cfg->numel, cfg->numel + cfg->num_tensors);
         ctx->last_grads.assign(static_cast<size_t>(nptr), nullptr);
         for (int32_t k = 0; k < cfg->num_tensors; ++k)
-            for (int64_t s = 0; s < cfg->numel[k]; s += desloc::CHUNK_ELEMS) {
+            for (int64_t s = 0; s < cfg->numel[k]; s += chunk_elems) {
                 desloc::Chunk ch;
                 ch.tensor = k;
                 ch.start = s;
                 const int64_t left = cfg->numel[k] - s;
-                ch.count = static_cast<int32_t>(left < desloc::CHUNK_ELEMS ? left : desloc::CHUNK_ELEMS);
+                ch.count = static_cast<int32_t>(left < chunk_elems ? left : chunk_elems);
                 chunks.push_back(ch);
             }
     } catch (const std::bad_alloc &) {
