@@ -441,10 +441,12 @@ def run_e2e(args, w, eng, G, X, offs, dev, world, barrier):
     steps = max(2, min(args.steps, 6))
     t_next = 1000
 
+    hv = views(H)
+
     def one(t):
-        for m in range(w.M):
-            G[m].copy_(H[m], non_blocking=True)
-        eng.step(t, w.lr, gv, clip_bound=w.clip_bound(t))
+        # desloc_step_host: the C-ABI call that takes HOST gradient buffers, copies them group by
+        # group and pipelines the step behind the copies; then the result read-back
+        eng.step_host(t, w.lr, hv, gv, clip_bound=w.clip_bound(t))
         out.copy_(X[0][last[0]:last[0] + last[1]], non_blocking=True)
         stream.synchronize()
 
@@ -465,7 +467,8 @@ def run_e2e(args, w, eng, G, X, offs, dev, world, barrier):
     return {"value": world * w.M * w.N * steps / (ms * 1e-3) / 1e9, "unit": UNIT,
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": last[1] * 4, "steps": steps,
             "ms_per_step": ms / steps,
-            "note": "gradients copied from pinned host memory every step"
+            "note": "desloc_step_host: gradients copied from pinned host memory every step, "
+                    "pipelined with the step in 8 tensor groups; result slice read back"
                     + ("" if share else " (one host buffer re-sent for each worker)")}
 
 

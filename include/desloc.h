@@ -140,6 +140,23 @@ DESLOC_API int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *
 DESLOC_API int desloc_step(desloc_ctx *ctx, int64_t t, float lr_t, float clip_bound_t,
                 const void *const *grads, void *stream, uint32_t *mask_out);
 
+/*
+ * desloc_step() for gradients that arrive in HOST memory (e.g. produced elsewhere and handed
+ * over through pinned buffers): same step, with the host-to-device copies inside the call.
+ *   host_grads : host array of M*num_tensors HOST pointers (page-locked memory if the copies
+ *                are to overlap with compute), same indexing and dtype as for desloc_step().
+ *   dev_grads  : host array of M*num_tensors DEVICE pointers to caller-owned staging buffers
+ *                of the same sizes; they receive the copies and are what the kernels read.
+ * The tensor list is cut into up to 8 groups; each group's gradients are copied on a stream
+ * the context owns (tensors adjacent in both host and device memory go as one copy) and the
+ * group's part of the step is launched on `stream` as soon as its copies have landed, so all
+ * but the last group's compute hides behind the transfers.  The copies wait for work already
+ * enqueued on `stream`.  Not available under stream capture (DESLOC_E_INVALID).
+ */
+DESLOC_API int desloc_step_host(desloc_ctx *ctx, int64_t t, float lr_t, float clip_bound_t,
+                                const void *const *host_grads, void *const *dev_grads,
+                                void *stream, uint32_t *mask_out);
+
 /* As desloc_step() but with the sync mask given by the caller instead of derived from t
    (used to time or test one sync pattern in isolation).  mask bits outside X|U|V, or V for
    SGDM, are rejected with DESLOC_E_INVALID.  Counters are updated as for desloc_step(). */

@@ -74,6 +74,9 @@ _lib.desloc_create.argtypes = [ctypes.POINTER(_P), ctypes.POINTER(DeslocConfig),
 _lib.desloc_step.restype = ctypes.c_int
 _lib.desloc_step.argtypes = [_P, ctypes.c_int64, ctypes.c_float, ctypes.c_float, _PP, _P,
                              ctypes.POINTER(ctypes.c_uint32)]
+_lib.desloc_step_host.restype = ctypes.c_int
+_lib.desloc_step_host.argtypes = [_P, ctypes.c_int64, ctypes.c_float, ctypes.c_float, _PP, _PP, _P,
+                                  ctypes.POINTER(ctypes.c_uint32)]
 _lib.desloc_step_masked.restype = ctypes.c_int
 _lib.desloc_step_masked.argtypes = [_P, ctypes.c_uint32, ctypes.c_float, ctypes.c_float, _PP, _P]
 _lib.desloc_destroy.restype = ctypes.c_int
@@ -162,6 +165,20 @@ def desloc_step(ctx: int, t: int, lr_t: float, clip_bound_t: float, grads, strea
                           ctypes.byref(mask))
     if rc != DESLOC_OK:
         raise DeslocError(rc, "desloc_step", _lib.desloc_last_cuda_error(ctx))
+    return int(mask.value)
+
+
+def desloc_step_host(ctx: int, t: int, lr_t: float, clip_bound_t: float, host_grads, dev_grads,
+                     stream: int = 0) -> int:
+    """desloc_step() with gradients in host memory: copies them into the device staging buffers
+    `dev_grads` group by group and pipelines the step behind the copies.  Returns the mask."""
+    hg = host_grads if isinstance(host_grads, ctypes.Array) else _ptr_array(host_grads)
+    dg = dev_grads if isinstance(dev_grads, ctypes.Array) else _ptr_array(dev_grads)
+    mask = ctypes.c_uint32(0)
+    rc = _lib.desloc_step_host(ctx, int(t), float(lr_t), float(clip_bound_t), hg, dg,
+                               stream or None, ctypes.byref(mask))
+    if rc != DESLOC_OK:
+        raise DeslocError(rc, "desloc_step_host", _lib.desloc_last_cuda_error(ctx))
     return int(mask.value)
 
 

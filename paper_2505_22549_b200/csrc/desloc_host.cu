@@ -39,6 +39,7 @@ const void *lookup_step_kernel(int opt, bool post, bool bf16, int mt, int mask) 
 namespace {
 
 constexpr int kSlots = 8;  // staging slots for per-step gradient pointer tables
+constexpr int kHostGroups = 8;  // pipeline depth of desloc_step_host
 
 struct Slot {
     void **host = nullptr;  // pinned
@@ -120,6 +121,15 @@ struct desloc_ctx {
     int64_t launches = 0;
     int last_cuda_error = 0;
     int ctas_per_sm = 0;  // 0: one block per work item; > 0: persistent grid of that many per SM
+    // desloc_step_host: tensor groups whose copies and kernels are pipelined
+    struct Group {
+        int32_t k0, k1;   // tensors [k0, k1)
+        int64_t c0, c1;   // chunks  [c0, c1)
+    };
+    std::vector<Group> groups;
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_entry = nullptr;
+    cudaEvent_t ev_group[kHostGroups] = {};
 };
 
 namespace {
@@ -165,6 +175,10 @@ uint32_t mask_at(const desloc_config *c, int64_t t) {
 void free_ctx(desloc_ctx *ctx) {
     if (!ctx) return;
     free_worker_res(ctx->res);
+    if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+    if (ctx->ev_entry) cudaEventDestroy(ctx->ev_entry);
+    for (cudaEvent_t ev : ctx->ev_group)
+        if (ev) cudaEventDestroy(ev);
     if (ctx->d_chunks) cudaFree(ctx->d_chunks);
     delete ctx;
 }
@@ -196,8 +210,12 @@ int stage_grads(desloc_ctx *ctx, const void *const *grads, cudaStream_t stream, 
 }
 
 // max_norm > 0: norm-based clipping first (two reduction launches), then the step.
+// host_grads != nullptr: the gradients are first copied from host memory into `grads` (device),
+// tensor group by tensor group on the context's copy stream, each group's kernel starting as
+// soon as its copies have landed.
 int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
-             const void *const *grads, cudaStream_t stream, float max_norm = 0.f) {
+             const void *const *grads, cudaStream_t stream, float max_norm = 0.f,
+             const void *const *host_grads = nullptr) {
     const desloc_config &c = ctx->cfg;
     if (!std::isfinite(lr_t) || std::isnan(max_norm)) return DESLOC_E_RANGE;
     const bool nclip = (c.flags & DESLOC_FLAG_ADOPT_NORM_CLIP) != 0;
@@ -223,6 +241,10 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
             break;
         }
         const bool capturing = cap != cudaStreamCaptureStatusNone;
+        if (capturing && host_grads) {
+            rc = DESLOC_E_INVALID;
+            break;
+        }
         void **d_g = nullptr;
         bool inline_g = false;
         if (!capturing) {
@@ -300,13 +322,60 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
         if (grid > 0x7fffffffLL) grid = 0x7fffffffLL;  // the kernel strides over the rest
         int kmask_arg = static_cast<int>(kmask);
         void *params[] = {&a, &kmask_arg};  // the second one is read by the generic kernel only
-        e = cudaLaunchKernel(fn, dim3(static_cast<unsigned>(grid)), dim3(desloc::BLOCK_THREADS),
-                             params, 0, stream);
+        if (!host_grads) {
+            e = cudaLaunchKernel(fn, dim3(static_cast<unsigned>(grid)), dim3(desloc::BLOCK_THREADS),
+                                 params, 0, stream);
+            if (e == cudaSuccess) ctx->launches += 1;
+        } else {
+            // The device gradient buffers may still be read by earlier work on `stream`.
+            const size_t gsz = c.grad_dtype == DESLOC_BF16 ? 2 : 4;
+            e = cudaEventRecord(ctx->ev_entry, stream);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_entry, 0);
+            for (size_t gi = 0; gi < ctx->groups.size() && e == cudaSuccess; ++gi) {
+                const desloc_ctx::Group &grp = ctx->groups[gi];
+                for (int m = 0; m < c.M && e == cudaSuccess; ++m) {
+                    // merge tensors that are adjacent on both sides into one copy
+                    int32_t k = grp.k0;
+                    while (k < grp.k1 && e == cudaSuccess) {
+                        const int64_t i0 = static_cast<int64_t>(m) * c.num_tensors + k;
+                        const char *hp = static_cast<const char *>(host_grads[i0]);
+                        char *dp = static_cast<char *>(const_cast<void *>(grads[i0]));
+                        size_t bytes = static_cast<size_t>(ctx->numel[k]) * gsz;
+                        int32_t k2 = k + 1;
+                        while (k2 < grp.k1) {
+                            const int64_t i2 = static_cast<int64_t>(m) * c.num_tensors + k2;
+                            if (static_cast<const char *>(host_grads[i2]) != hp + bytes ||
+                                static_cast<const char *>(grads[i2]) != dp + bytes)
+                                break;
+                            bytes += static_cast<size_t>(ctx->numel[k2]) * gsz;
+                            ++k2;
+                        }
+                        e = cudaMemcpyAsync(dp, hp, bytes, cudaMemcpyHostToDevice, ctx->copy_stream);
+                        k = k2;
+                    }
+                }
+                if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_group[gi], ctx->copy_stream);
+                if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->ev_group[gi], 0);
+                if (e != cudaSuccess) break;
+                a.chunks = ctx->d_chunks + grp.c0;
+                a.nchunks = grp.c1 - grp.c0;
+                const long long items =
+                    per_worker_items
+                        ? ((a.nchunks + desloc::LOCAL_SLOTS - 1) / desloc::LOCAL_SLOTS) * c.M
+                        : a.nchunks;
+                long long ggrid = items;
+                if (ctx->ctas_per_sm > 0 && ggrid > static_cast<long long>(ctx->ctas_per_sm) * ctx->num_sms)
+                    ggrid = static_cast<long long>(ctx->ctas_per_sm) * ctx->num_sms;
+                if (ggrid > 0x7fffffffLL) ggrid = 0x7fffffffLL;
+                e = cudaLaunchKernel(fn, dim3(static_cast<unsigned>(ggrid)),
+                                     dim3(desloc::BLOCK_THREADS), params, 0, stream);
+                if (e == cudaSuccess) ctx->launches += 1;
+            }
+        }
         if (e != cudaSuccess) {
             rc = cuda_fail(ctx, e);
             break;
         }
-        ctx->launches += 1;
         if (!capturing) {
             Slot &s = ctx->res.slots[ctx->cur_slot];
             e = cudaEventRecord(s.done, stream);
@@ -418,8 +487,28 @@ int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *const *x, f
     if (e == cudaSuccess)
         e = cudaMemcpy(ctx->d_chunks, chunks.data(), chunks.size() * sizeof(desloc::Chunk),
                        cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_entry, cudaEventDisableTiming);
+    for (int i = 0; i < kHostGroups && e == cudaSuccess; ++i)
+        e = cudaEventCreateWithFlags(&ctx->ev_group[i], cudaEventDisableTiming);
     if (e == cudaSuccess) {
         try {
+            // tensor groups of about equal size for desloc_step_host
+            int64_t c = 0, acc = 0;
+            int32_t k0 = 0;
+            int64_t c0 = 0;
+            for (int32_t k = 0; k < cfg->num_tensors; ++k) {
+                c += (cfg->numel[k] + chunk_elems - 1) / chunk_elems;
+                acc += cfg->numel[k];
+                const int done_groups = static_cast<int>(ctx->groups.size());
+                const bool last = k == cfg->num_tensors - 1;
+                if (last || (done_groups < kHostGroups - 1 &&
+                             acc * kHostGroups >= total * (done_groups + 1))) {
+                    ctx->groups.push_back({k0, k + 1, c0, c});
+                    k0 = k + 1;
+                    c0 = c;
+                }
+            }
             e = make_worker_res(ctx->res, cfg->M, cfg->num_tensors, ctx->nchunks,
                                 cfg->opt != DESLOC_SGDM, x, u, v);
         } catch (const std::bad_alloc &) {
@@ -442,6 +531,21 @@ int desloc_step(desloc_ctx *ctx, int64_t t, float lr_t, float clip_bound_t,
     if (t < 0) return DESLOC_E_RANGE;
     const uint32_t mask = mask_at(&ctx->cfg, t);
     const int rc = run_step(ctx, mask, lr_t, clip_bound_t, grads, static_cast<cudaStream_t>(stream));
+    if (rc == DESLOC_OK && mask_out) *mask_out = mask;
+    return rc;
+}
+
+int desloc_step_host(desloc_ctx *ctx, int64_t t, float lr_t, float clip_bound_t,
+                     const void *const *host_grads, void *const *dev_grads, void *stream,
+                     uint32_t *mask_out) {
+    if (!ctx || !host_grads || !dev_grads) return DESLOC_E_NULL;
+    if (t < 0) return DESLOC_E_RANGE;
+    for (int64_t i = 0; i < ctx->nptr; ++i)
+        if (!host_grads[i]) return DESLOC_E_NULL;
+    const uint32_t mask = mask_at(&ctx->cfg, t);
+    const int rc = run_step(ctx, mask, lr_t, clip_bound_t,
+                            reinterpret_cast<const void *const *>(dev_grads),
+                            static_cast<cudaStream_t>(stream), 0.f, host_grads);
     if (rc == DESLOC_OK && mask_out) *mask_out = mask;
     return rc;
 }

@@ -101,6 +101,19 @@ class DesLoc:
         self.M = M
         self._gkey = self._garr = None
 
+    def step_host(self, t: int, lr: float, host_grads, dev_grads, clip_bound: float = 0.0) -> int:
+        """Step t with gradients in (pinned) host tensors; dev_grads are device staging tensors."""
+        want = torch.bfloat16 if self.grad_dtype == B.DESLOC_BF16 else torch.float32
+        hp = []
+        for lst in host_grads:
+            for t_, n in zip(lst, self.numel):
+                if t_.dtype != want or t_.numel() != n or not t_.is_contiguous() or t_.is_cuda:
+                    raise ValueError("host gradient tensor of wrong dtype, size, layout or device")
+                hp.append(t_.data_ptr())
+        stream = torch.cuda.current_stream(self.device).cuda_stream
+        return B.desloc_step_host(self.ctx, t, lr, clip_bound, hp, self._grad_array(dev_grads),
+                                  stream)
+
     def step_masked(self, mask: int, lr: float, grads, clip_bound: float = 0.0) -> None:
         stream = torch.cuda.current_stream(self.device).cuda_stream
         B.desloc_step_masked(self.ctx, mask, lr, clip_bound, self._grad_array(grads), stream)

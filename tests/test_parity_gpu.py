@@ -255,6 +255,37 @@ def test_gradient_pointers_may_change_every_step_and_lr_schedule():
     eng.close()
 
 
+@pytest.mark.parametrize("name", ["cfg2_adam_135m", "cfg3_adopt_360m"])
+def test_step_host_equals_step_with_device_gradients(name):
+    """Gradients handed over in pinned host memory: same bits as the device-gradient path, for
+    packed buffers (merged copies) and for separately allocated tensors."""
+    d = _lib()
+    w = di.mini(di.WORKLOADS[name], T=6).replace(K=(2, 3, 4))
+    dev = torch.device("cuda:0")
+    a, b = State(w, dev), State(w, dev)
+    ea, eb = make_engine(d, w, a), make_engine(d, w, b)
+    hflat = [torch.empty(b.nflat, dtype=b.g[0].dtype).pin_memory() for _ in range(w.M)]
+    hsep = [[torch.empty(n, dtype=b.g[0].dtype).pin_memory() for n in w.numel] for _ in range(w.M)]
+    hview = [[h[o:o + n] for o, n in zip(b.offs, w.numel)] for h in hflat]
+    for t in range(w.T):
+        a.fill_grads(t)
+        for m in range(w.M):
+            hflat[m].copy_(a.g[m])
+            for hs, src in zip(hsep[m], a.views(a.g)[m]):
+                hs.copy_(src)
+            b.g[m].zero_()
+        torch.cuda.synchronize()
+        lr, cb = f32r(w.lr), f32r(w.clip_bound(t))
+        ma = ea.step(t, lr, a.views(a.g), clip_bound=cb)
+        mb = eb.step_host(t, lr, hview if t % 2 == 0 else hsep, b.views(b.g), clip_bound=cb)
+        assert ma == mb
+    torch.cuda.synchronize()
+    for pa, pb in [(a.x, b.x), (a.u, b.u), (a.v, b.v)]:
+        assert np.array_equal(a.to_numpy(pa), b.to_numpy(pb))
+    assert eb.launches() > ea.launches()      # one launch per tensor group
+    ea.close(); eb.close()
+
+
 def test_errors_are_status_codes_and_context_survives():
     d = _lib()
     dev = torch.device("cuda:0")
