@@ -24,6 +24,11 @@
 #ifndef DESLOC_SPLIT_LARGE_M
 #define DESLOC_SPLIT_LARGE_M 1
 #endif
+// 1: hardware reciprocal square root (about 2 ulp) instead of IEEE sqrt + division in the Adam
+// direction and the ADOPT normaliser.
+#ifndef DESLOC_FAST_MATH
+#define DESLOC_FAST_MATH 0
+#endif
 #ifndef DESLOC_MINB_LARGE_M
 #define DESLOC_MINB_LARGE_M 3
 #endif
@@ -156,7 +161,11 @@ __device__ __forceinline__ void state_update(const StepArgs &a, float g, float u
         vn = fmaf(a.b2, vp, (a.omb2 * gh) * gh);
     } else if constexpr (OPT == OPT_ADOPT) {
         vn = fmaf(a.b2, vp, (a.omb2 * gh) * gh);
+#if DESLOC_FAST_MATH
+        float r = gh * rsqrtf(fmaxf(vown, a.eps * a.eps));
+#else
         float r = gh / fmaxf(sqrtf(vown), a.eps);
+#endif
         r = fminf(fmaxf(r, -a.cbound), a.cbound);
         un = fmaf(a.b1, up, a.omb1 * r);
     } else {
@@ -169,10 +178,15 @@ __device__ __forceinline__ void state_update(const StepArgs &a, float g, float u
 template <int OPT>
 __device__ __forceinline__ float param_step(const StepArgs &a, float xp, float un, float vn) {
     float d;
-    if constexpr (OPT == OPT_ADAM)
+    if constexpr (OPT == OPT_ADAM) {
+#if DESLOC_FAST_MATH
+        d = (a.lr * un) * rsqrtf(vn + a.lam2);
+#else
         d = (a.lr * un) / sqrtf(vn + a.lam2);
-    else
+#endif
+    } else {
         d = a.lr * un;
+    }
     // x* (1 - eta wd) - d, written as x* - (eta wd x* + d): one rounding at x's scale
     return xp - fmaf(a.lrwd, xp, d);
 }

@@ -26,52 +26,116 @@ __device__ __forceinline__ float block_sum(float v, float *warp_sums) {
     return t;  // valid in thread 0
 }
 
-// partial[m * nchunks + c] = sum over chunk c of g^m squared.  Work item = (worker, chunk).
+// partial[m * ngroups + q] = sum of g^m squared over chunk group q (SUMSQ_GROUP consecutive
+// chunks).  Work item = (worker, group): a block streams up to 64 KB of one worker's gradient
+// with eight independent loads per thread in flight, and reduces once.
+constexpr int SUMSQ_GROUP = 8;
+
 template <typename GT>
-__global__ void __launch_bounds__(BLOCK_THREADS, 6)
+__device__ __forceinline__ float chunk_sumsq(const Chunk &ch, const void *const *g, int nt, int m,
+                                             float acc) {
+    const int tid = threadIdx.x;
+    const char *base = reinterpret_cast<const char *>(g[static_cast<long long>(m) * nt + ch.tensor]) +
+                       ch.start * static_cast<long long>(sizeof(GT));
+    const bool aligned = (reinterpret_cast<uintptr_t>(base) & (sizeof(GT) == 2 ? 7u : 15u)) == 0;
+    if (aligned) {
+        const int n4 = ch.count >> 2;
+        FV<4> v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int p = tid + j * BLOCK_THREADS;
+            if (p < n4) v[j] = ld_grad<4, GT>(base, static_cast<long long>(p) * 4);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int p = tid + j * BLOCK_THREADS;
+            if (p < n4) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) acc = fmaf(v[j].a[k], v[j].a[k], acc);
+            }
+        }
+        const int rem = ch.count & 3;
+        if (tid < rem) {
+            const float t = ld_grad<1, GT>(base, (n4 << 2) + tid).a[0];
+            acc = fmaf(t, t, acc);
+        }
+    } else {
+        for (int e = tid; e < ch.count; e += BLOCK_THREADS) {
+            const float t = ld_grad<1, GT>(base, e).a[0];
+            acc = fmaf(t, t, acc);
+        }
+    }
+    return acc;
+}
+
+// Eight bf16 values in one 128-bit load.
+__device__ __forceinline__ float sumsq8_bf16(const uint4 &t, float acc) {
+    const unsigned w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float lo = __uint_as_float(w[k] << 16), hi = __uint_as_float(w[k] & 0xffff0000u);
+        acc = fmaf(lo, lo, acc);
+        acc = fmaf(hi, hi, acc);
+    }
+    return acc;
+}
+
+template <typename GT>
+__global__ void __launch_bounds__(BLOCK_THREADS, 8)
 sumsq_kernel(const Chunk *chunks, long long nchunks, const void *const *g, int nt, int M,
              float *partial) {
     __shared__ float warp_sums[BLOCK_THREADS / 32];
-    const long long nitems = nchunks * M;
+    const long long ngroups = (nchunks + SUMSQ_GROUP - 1) / SUMSQ_GROUP;
+    const long long nitems = ngroups * M;
     const int tid = threadIdx.x;
     for (long long item = blockIdx.x; item < nitems; item += gridDim.x) {
-        const long long c = item % nchunks;
-        const int m = static_cast<int>(item / nchunks);
-        const Chunk ch = chunks[c];
-        const char *base = reinterpret_cast<const char *>(g[static_cast<long long>(m) * nt + ch.tensor]) +
-                           ch.start * static_cast<long long>(sizeof(GT));
-        const bool aligned = (reinterpret_cast<uintptr_t>(base) & (sizeof(GT) == 2 ? 7u : 15u)) == 0;
-        float acc = 0.f;
-        if (aligned) {
-            const int n4 = ch.count >> 2;
-            FV<4> v[4];
-            // up to four independent 128/64-bit loads per thread before the first use
+        const long long q = item % ngroups;
+        const int m = static_cast<int>(item / ngroups);
+        const long long c0 = q * SUMSQ_GROUP;
+        float acc0 = 0.f, acc1 = 0.f;
+        // four chunks per iteration; full, 16-byte aligned bf16 chunks take the wide path with
+        // all eight 128-bit loads of the iteration issued before the first use
+#pragma unroll 1
+        for (int k = 0; k < SUMSQ_GROUP; k += 4) {
+            if constexpr (sizeof(GT) == 2) {
+                uint4 r[4][2];
+                bool wide[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int p = tid + j * BLOCK_THREADS;
-                if (p < n4) v[j] = ld_grad<4, GT>(base, static_cast<long long>(p) * 4);
-            }
+                for (int j = 0; j < 4; ++j) {
+                    wide[j] = false;
+                    if (c0 + k + j < nchunks) {
+                        const Chunk ch = chunks[c0 + k + j];
+                        const char *base =
+                            reinterpret_cast<const char *>(g[static_cast<long long>(m) * nt + ch.tensor]) +
+                            ch.start * 2;
+                        wide[j] = ch.count == CHUNK_ELEMS && (reinterpret_cast<uintptr_t>(base) & 15u) == 0;
+                        if (wide[j]) {
+                            const uint4 *p = reinterpret_cast<const uint4 *>(base);
+                            r[j][0] = __ldcs(p + tid);
+                            r[j][1] = __ldcs(p + tid + BLOCK_THREADS);
+                        }
+                    }
+                }
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int p = tid + j * BLOCK_THREADS;
-                if (p < n4) {
+                for (int j = 0; j < 4; ++j) {
+                    if (wide[j]) {
+                        acc0 = sumsq8_bf16(r[j][0], acc0);
+                        acc1 = sumsq8_bf16(r[j][1], acc1);
+                    } else if (c0 + k + j < nchunks) {
+                        acc0 = chunk_sumsq<GT>(chunks[c0 + k + j], g, nt, m, acc0);
+                    }
+                }
+            } else {
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) acc = fmaf(v[j].a[k], v[j].a[k], acc);
+                for (int j = 0; j < 4; j += 2) {
+                    if (c0 + k + j < nchunks) acc0 = chunk_sumsq<GT>(chunks[c0 + k + j], g, nt, m, acc0);
+                    if (c0 + k + j + 1 < nchunks)
+                        acc1 = chunk_sumsq<GT>(chunks[c0 + k + j + 1], g, nt, m, acc1);
                 }
             }
-            const int rem = ch.count & 3;
-            if (tid < rem) {
-                const float t = ld_grad<1, GT>(base, (n4 << 2) + tid).a[0];
-                acc = fmaf(t, t, acc);
-            }
-        } else {
-            for (int e = tid; e < ch.count; e += BLOCK_THREADS) {
-                const float t = ld_grad<1, GT>(base, e).a[0];
-                acc = fmaf(t, t, acc);
-            }
         }
-        const float total = block_sum(acc, warp_sums);
-        if (tid == 0) partial[static_cast<long long>(m) * nchunks + c] = total;
+        const float total = block_sum(acc0 + acc1, warp_sums);
+        if (tid == 0) partial[static_cast<long long>(m) * ngroups + q] = total;
     }
 }
 
@@ -193,14 +257,15 @@ unsigned grid_for(long long nitems) {
 cudaError_t launch_grad_norms(const Chunk *chunks, long long nchunks, const void *const *g, int nt,
                               int M, bool bf16, float max_norm, float *partial, float *norms,
                               float *scales, cudaStream_t stream) {
-    const unsigned grid = grid_for(nchunks * M);
+    const long long ngroups = (nchunks + SUMSQ_GROUP - 1) / SUMSQ_GROUP;
+    const unsigned grid = grid_for(ngroups * M);
     if (bf16)
         sumsq_kernel<bf16_t><<<grid, BLOCK_THREADS, 0, stream>>>(chunks, nchunks, g, nt, M, partial);
     else
         sumsq_kernel<float><<<grid, BLOCK_THREADS, 0, stream>>>(chunks, nchunks, g, nt, M, partial);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    norm_finalize_kernel<<<M, BLOCK_THREADS, 0, stream>>>(partial, nchunks, max_norm, norms, scales);
+    norm_finalize_kernel<<<M, BLOCK_THREADS, 0, stream>>>(partial, ngroups, max_norm, norms, scales);
     return cudaGetLastError();
 }
 
