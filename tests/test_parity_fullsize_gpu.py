@@ -64,8 +64,42 @@ def test_fullsize_sampled_parity(name, T, t0, nsamp):
         frac_exact = float(np.mean(got == ref))
         print(f"{name} {nm}: max rel err {max(rel_err(got[m], ref[m]) for m in range(w.M)):.2e}, "
               f"bit-exact {100 * frac_exact:.2f}%")
-    # untouched neighbours: the sampled set covers the last 64 elements of each tensor, and the
-    # padding between tensors (if any) must still be zero
+    eng.close()
+    del st, eng
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("name", ["cfg5_adam_ddp", "cfg5_sgdm_local"])
+def test_fullsize_identical_gradients_keep_replicas_bitwise_equal(name):
+    """Workload 5's identical-gradient run at full size (361.8 M parameters x 8 workers): with the
+    same gradient on every worker the replicas must stay bitwise equal to one another under any
+    schedule -- a property that holds at any size and needs no oracle -- and, on sampled
+    coordinates, equal to the oracle's single-worker run."""
+    import paper_2505_22549_b200 as d
+    w = di.WORKLOADS[name]
+    dev = torch.device("cuda:0")
+    free, _ = torch.cuda.mem_get_info()
+    if free < w.N * w.M * 14 + (6 << 30):
+        pytest.skip("not enough device memory")
+    st = State(w, dev, align=4)
+    eng = make_engine(d, w, st)
+    idx_np = di.sample_indices(w.numel, 1 << 14, seed=3, align=4)
+    idx = torch.from_numpy(idx_np).to(dev)
+    one = w.replace(M=1)
+    ox, ou = st.to_numpy(st.x[:1], idx), st.to_numpy(st.u[:1], idx)
+    ov = st.to_numpy(st.v[:1], idx) if st.v is not None else None
+    gviews = st.views(st.g)
+    for t in range(17):                          # crosses t = 16 for the K = 16 schedule
+        di.fill_grads_(w, t, 0, st.g[0], align=4)
+        for m in range(1, w.M):
+            st.g[m].copy_(st.g[0])
+        eng.step(t, f32r(w.lr), gviews)
+        oracle.step(oracle_cfg(one), t, f32r(w.lr), ox, ou, ov, st.to_numpy(st.g[:1], idx))
+    torch.cuda.synchronize()
+    for bufs, ref in [(st.x, ox), (st.u, ou)] + ([(st.v, ov)] if ov is not None else []):
+        for m in range(1, w.M):
+            assert torch.equal(bufs[m], bufs[0]), f"replica {m} differs from replica 0"
+        assert rel_err(st.to_numpy(bufs[:1], idx)[0], ref[0]) <= TOL
     eng.close()
     del st, eng
     torch.cuda.empty_cache()

@@ -286,6 +286,87 @@ def test_step_host_equals_step_with_device_gradients(name):
     ea.close(); eb.close()
 
 
+def test_guard_bands_around_every_tensor_stay_untouched():
+    """Each element is written by exactly one thread and nothing outside a tensor is touched:
+    tensors are laid out with up to 15 elements of padding between them (and 32 in front and
+    behind), filled with a sentinel that must survive every kind of step."""
+    d = _lib()
+    SENT = -12288.0        # exact in bf16 too
+    for opt, M in [("adam", 4), ("adopt", 8), ("sgdm", 3), ("adam", 12), ("adam", 1)]:
+        numel = (1, 5, 4096, 4097, 777, 8192 + 3, 64)
+        w = di.Workload("guard", opt, M, numel, "bf16", "normal1", lr=1e-2, clip_rho=1.0, seed=9,
+                        adopt_norm_clip=(opt == "adopt"))
+        dev = torch.device("cuda:0")
+        offs, pos = [], 32
+        for n in numel:
+            pos = -(-pos // 16) * 16 + (4 if n % 2 else 0)   # some starts 16-byte aligned, some not
+            offs.append(pos)
+            pos += n + 5
+        total = pos + 32
+        mk = lambda dt: torch.full((total,), SENT, dtype=dt, device=dev)
+        X, U, V = [mk(torch.float32) for _ in range(M)], [mk(torch.float32) for _ in range(M)], \
+            [mk(torch.float32) for _ in range(M)]
+        G = [mk(torch.bfloat16) for _ in range(M)]
+        views = lambda bufs: [[b[o:o + n] for o, n in zip(offs, numel)] for b in bufs]
+        for bufs, val in ((X, 0.5), (U, 0.0), (V, 0.25), (G, 0.125)):
+            for lst in views(bufs):
+                for t in lst:
+                    t.fill_(val)
+        eng = d.DesLoc(views(X), views(U), views(V) if opt != "sgdm" else None, opt=opt,
+                       grad_dtype="bf16", clip_rho=1.0, K=(2, 3, 4),
+                       flags=d.DESLOC_FLAG_ADOPT_NORM_CLIP if opt == "adopt" else 0)
+        inside = torch.zeros(total, dtype=torch.bool, device=dev)
+        for o, n in zip(offs, numel):
+            inside[o:o + n] = True
+        for t in range(13):
+            if t % 3 == 2:
+                eng.step_normclip(t, 1e-2, views(G), 0.01, clip_bound=1.0)
+            else:
+                eng.step(t, 1e-2, views(G), clip_bound=1.0)
+        torch.cuda.synchronize()
+        for bufs in (X, U) + ((V,) if opt != "sgdm" else ()):
+            for b in bufs:
+                assert bool((b[~inside] == SENT).all()), f"{opt} M={M}: wrote outside a tensor"
+                assert bool((b[inside] != SENT).all())
+        assert bool((X[0][inside] != 0.5).all())          # every element was updated
+        for b in G:
+            assert bool((b[~inside].float() == SENT).all())
+        eng.close()
+
+
+def test_never_sync_periods_and_large_step_numbers():
+    """K = 0 means never (the FedAvg-with-local-states baseline keeps K_u = K_v = 0); t far
+    beyond 2^31 still schedules correctly."""
+    d = _lib()
+    w = di.Workload("never", "adam", 3, (100, 4096), "f32", "normal1", lr=1e-2, K=(4, 0, 0), seed=2)
+    res = run_both(w, 9)
+    check(res)
+    assert res["gpu_masks"] == [1, 0, 0, 0, 1, 0, 0, 0, 1]
+    assert res["counters"] == [9, 3, 0, 0]
+    dev = torch.device("cuda:0")
+    st = State(w.replace(K=(3, 5, 7)), dev)
+    eng = make_engine(d, w.replace(K=(3, 5, 7)), st)
+    st.fill_grads(0)
+    big = 3 * 5 * 7 * (1 << 40)
+    assert eng.step(big, 1e-3, st.views(st.g)) == 7
+    assert eng.step(big + 3, 1e-3, st.views(st.g)) == 1
+    assert eng.step(big + 35, 1e-3, st.views(st.g)) == 6
+    torch.cuda.synchronize()
+    eng.close()
+
+
+def test_create_on_a_device_that_does_not_exist():
+    d = _lib()
+    x = torch.zeros(4, device="cuda:0")
+    cfg = d.make_config(1, [4], "sgdm", "f32")
+    with pytest.raises(d.DeslocError) as e:
+        d.desloc_create(cfg, [x.data_ptr()], [x.data_ptr()], None, 4096)
+    assert e.value.status == d.DESLOC_E_CUDA
+    # the failed create left the runtime usable
+    ctx = d.desloc_create(cfg, [x.data_ptr()], [torch.zeros(4, device="cuda:0").data_ptr()], None, 0)
+    d.desloc_destroy(ctx)
+
+
 def test_errors_are_status_codes_and_context_survives():
     d = _lib()
     dev = torch.device("cuda:0")
