@@ -41,7 +41,7 @@
 extern "C" {
 #endif
 
-#define DESLOC_MAX_M 64 /* largest worker count a context accepts */
+#define DESLOC_MAX_M 256 /* largest worker count a context accepts (the toy problem of the paper uses 256) */
 
 typedef struct desloc_ctx desloc_ctx; /* opaque, library-owned */
 

@@ -23,7 +23,7 @@ DESLOC_OK, DESLOC_E_NULL, DESLOC_E_RANGE, DESLOC_E_INVALID, DESLOC_E_NOMEM, DESL
     0, -1, -2, -3, -4, -5
 DESLOC_E_TOO_LARGE = -6
 DESLOC_STATIC_MAX_POINTERS, DESLOC_STATIC_MAX_CHUNKS = 2048, 16384
-DESLOC_MAX_M = 64
+DESLOC_MAX_M = 256
 
 OPT_BY_NAME = {"adam": DESLOC_ADAM, "adopt": DESLOC_ADOPT, "sgdm": DESLOC_SGDM}
 DTYPE_BY_NAME = {"f32": DESLOC_F32, "bf16": DESLOC_BF16}

@@ -72,7 +72,7 @@ def test_workload_sizes_match_the_stated_totals():
 
 
 BAD = [
-    (dict(M=0), "DESLOC_E_RANGE"), (dict(M=65), "DESLOC_E_RANGE"),
+    (dict(M=0), "DESLOC_E_RANGE"), (dict(M=257), "DESLOC_E_RANGE"),
     (dict(Kx=-1), "DESLOC_E_RANGE"), (dict(beta1=1.0), "DESLOC_E_RANGE"),
     (dict(beta2=-0.1), "DESLOC_E_RANGE"), (dict(beta1=float("nan")), "DESLOC_E_RANGE"),
     (dict(eps=-1.0), "DESLOC_E_RANGE"), (dict(weight_decay=-1.0), "DESLOC_E_RANGE"),

@@ -100,7 +100,7 @@ def test_set_workers_rejects_bad_arguments():
     cfg = d.make_config(2, [8], "adam", "f32")
     p = [b.data_ptr() for b in bufs]
     ctx = d.desloc_create(cfg, p[0:2], p[2:4], p[4:6], 0)
-    for M_new, first in [(0, 0), (65, 0), (2, 3), (2, -1)]:
+    for M_new, first in [(0, 0), (257, 0), (2, 3), (2, -1)]:
         with pytest.raises(d.DeslocError) as e:
             d.desloc_set_workers(ctx, M_new, first, p[0:2], p[2:4], p[4:6])
         assert e.value.status == d.DESLOC_E_RANGE

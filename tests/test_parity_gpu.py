@@ -129,7 +129,7 @@ def test_post_average_ordering(opt, M):
 
 
 @pytest.mark.parametrize("opt", ["adam", "adopt", "sgdm"])
-@pytest.mark.parametrize("M,post", [(9, False), (16, False), (16, True), (33, True), (64, False)])
+@pytest.mark.parametrize("M,post", [(9, False), (16, False), (16, True), (33, True), (64, False), (256, False)])
 def test_many_workers_runtime_m_path(opt, M, post):
     """More workers than the register-resident kernels hold (M > 8): runtime-M kernel on sync
     steps, per-worker items on local steps; up to the largest M a context accepts."""
