@@ -132,7 +132,10 @@ DESLOC_API int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *
  * Stream capture (CUDA graphs, for small launch-bound problems): the call may be made while
  * `stream` is capturing if either M*num_tensors <= 32 (the gradient pointers then travel in
  * the kernel parameters) or `grads` holds the same pointers as the previous, un-captured call
- * on that stream; otherwise it returns DESLOC_E_INVALID and captures nothing.  t, lr_t and
+ * on that stream; otherwise it returns DESLOC_E_INVALID and captures nothing.  (In the second
+ * case the captured launch refers to the context's staging slot of that pointer set, which is
+ * recycled after eight later un-captured calls with other gradient pointers: replay the graph
+ * only while fewer than eight such calls have been made.)  t, lr_t and
  * clip_bound_t are frozen into the captured launch, so a replayed graph repeats the same mask
  * sequence: capture a window of lcm(Kx, Ku, Kv) steps starting at a multiple of it.  Counters
  * and the launch count advance when a call is captured, not when the graph is replayed.

@@ -250,17 +250,16 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
         if (!capturing) {
             rc = stage_grads(ctx, grads, stream, &d_g);
             if (rc != DESLOC_OK) break;
+        } else if (ctx->nptr <= desloc::INLINE_PTRS && max_norm <= 0.f) {
+            inline_g = true;  // pointers travel in the kernel parameters: nothing to keep alive
         } else if (ctx->cur_slot >= 0 && stream == ctx->last_stream &&
                    std::memcmp(ctx->last_grads.data(), grads,
                                static_cast<size_t>(ctx->nptr) * sizeof(void *)) == 0) {
-            d_g = ctx->res.slots[ctx->cur_slot].dev;  // table already resident
-        } else if (ctx->nptr <= desloc::INLINE_PTRS && max_norm <= 0.f) {
-            inline_g = true;  // pointers travel in the kernel parameters
+            d_g = ctx->res.slots[ctx->cur_slot].dev;  // table already resident in this slot
         } else {
             rc = DESLOC_E_INVALID;  // stage these pointers with one un-captured step first
             break;
         }
-
         const float *d_gscale = nullptr;
         if (max_norm > 0.f) {
             e = desloc::launch_grad_norms(ctx->d_chunks, ctx->nchunks,

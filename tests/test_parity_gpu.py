@@ -367,6 +367,35 @@ def test_create_on_a_device_that_does_not_exist():
     d.desloc_destroy(ctx)
 
 
+def test_two_contexts_on_two_streams_and_stream_changes():
+    """Independent contexts may run concurrently on different streams; one context may move from
+    stream to stream (its gradient pointer table is re-staged on the new stream).  Results equal
+    the plain single-stream runs bit for bit."""
+    d = _lib()
+    dev = torch.device("cuda:0")
+    wa = di.mini(di.WORKLOADS["cfg2_adam_135m"], T=8).replace(K=(2, 3, 4))
+    wb = di.mini(di.WORKLOADS["cfg5_sgdm_desloc"], T=8).replace(K=(3, 2, 0), seed=4)
+    ref_a, ref_b = run_both(wa, wa.T), run_both(wb, wb.T)
+    sa, sb = State(wa, dev), State(wb, dev)
+    ea, eb = make_engine(d, wa, sa), make_engine(d, wb, sb)
+    streams = [torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()]
+    torch.cuda.synchronize()
+    for t in range(8):
+        sa.fill_grads(t)
+        sb.fill_grads(t)
+        torch.cuda.synchronize()                       # gradients ready before the side streams read them
+        with torch.cuda.stream(streams[t % 2]):        # context a hops between two streams
+            ea.step(t, f32r(wa.lr), sa.views(sa.g))
+        with torch.cuda.stream(streams[2]):            # context b runs alongside on a third
+            eb.step(t, f32r(wb.lr), sb.views(sb.g))
+        for s_ in streams:                             # a's next step must see this one's result
+            s_.synchronize()
+    torch.cuda.synchronize()
+    assert np.array_equal(sa.to_numpy(sa.x), ref_a["gx"]) and np.array_equal(sa.to_numpy(sa.v), ref_a["gv"])
+    assert np.array_equal(sb.to_numpy(sb.x), ref_b["gx"]) and np.array_equal(sb.to_numpy(sb.u), ref_b["gu"])
+    ea.close(); eb.close()
+
+
 def test_errors_are_status_codes_and_context_survives():
     d = _lib()
     dev = torch.device("cuda:0")
