@@ -236,6 +236,8 @@ def run_ours(args, w):
         di.fill_grads_(w.replace(seed=w.seed + rank), 0, m, G[m], align=align)
     views = lambda bufs: [[b[o:o + n] for o, n in zip(offs, w.numel)] for b in bufs]
     flags = d.DESLOC_FLAG_ADOPT_NORM_CLIP if w.adopt_norm_clip else 0
+    if args.post_average:
+        flags |= d.DESLOC_FLAG_POST_AVERAGE
     eng = d.DesLoc(views(X), views(U), views(V) if V is not None else None, opt=w.opt,
                    grad_dtype=w.grad_dtype, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
                    weight_decay=w.weight_decay, clip_rho=w.clip_rho, K=w.K, flags=flags)
@@ -391,6 +393,7 @@ def run_ours(args, w):
                        "l2": ("inputs larger than L2 (no flush needed)" if resident > (126 << 20)
                               else "workload fits in L2: latency-bound, see graph_window"),
                        "parallelism": f"{world} independent replica set(s), no collective",
+                       "ordering": "post-average" if args.post_average else "pre-average",
                        "masks_in_timed_region": masks},
             "roofline": roofline, "by_mask": by_mask, "normclip_step": normclip, "graph_window": graph_info, "cpu_baseline": {k: cpu[k] for k in
                                                                        ("value", "unit", "cores", "kind", "sample")},
@@ -482,6 +485,8 @@ def main():
     ap.add_argument("--ctas-per-sm", type=int, default=None)
     ap.add_argument("--workers", type=int, default=None,
                     help="override the workload's worker count M (exploration only)")
+    ap.add_argument("--post-average", action="store_true",
+                    help="average after the update (ordering of Algorithms 4-5) instead of before")
     ap.add_argument("--skip-e2e", action="store_true", help="omit the host-buffer leg (profiling)")
     ap.add_argument("--skip-cpu", action="store_true", help="omit the CPU oracle leg (profiling)")
     args = ap.parse_args()
