@@ -57,35 +57,39 @@ def build(force: bool = False) -> str:
     return _LIB
 
 
+def configure(L: ctypes.CDLL) -> ctypes.CDLL:
+    """Declare the argument and result types of every oracle entry point on a loaded library."""
+    L.desloc_oracle_sync_mask.restype = ctypes.c_uint32
+    L.desloc_oracle_sync_mask.argtypes = [ctypes.c_int32] * 4 + [ctypes.c_int64]
+    L.desloc_oracle_step.restype = ctypes.c_uint32
+    L.desloc_oracle_step.argtypes = [
+        ctypes.POINTER(OracleCfg), ctypes.c_int64, ctypes.c_double, ctypes.c_double,
+        ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+        ctypes.c_void_p]
+    L.desloc_oracle_step_scaled.restype = ctypes.c_uint32
+    L.desloc_oracle_step_scaled.argtypes = L.desloc_oracle_step.argtypes + [ctypes.c_void_p]
+    L.desloc_oracle_norm_scales.restype = None
+    L.desloc_oracle_norm_scales.argtypes = [ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
+                                            ctypes.c_void_p, ctypes.c_double, ctypes.c_void_p,
+                                            ctypes.c_void_p]
+    L.desloc_oracle_worker_mean.restype = None
+    L.desloc_oracle_worker_mean.argtypes = [ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
+                                            ctypes.c_void_p, ctypes.c_void_p]
+    L.desloc_oracle_rel_change.restype = None
+    L.desloc_oracle_rel_change.argtypes = [ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
+                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+    L.desloc_oracle_run.restype = None
+    L.desloc_oracle_run.argtypes = [
+        ctypes.POINTER(OracleCfg), ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p,
+        ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p,
+        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+    return L
+
+
 def lib() -> ctypes.CDLL:
     global _lib
     if _lib is None:
-        L = ctypes.CDLL(build())
-        L.desloc_oracle_sync_mask.restype = ctypes.c_uint32
-        L.desloc_oracle_sync_mask.argtypes = [ctypes.c_int32] * 4 + [ctypes.c_int64]
-        L.desloc_oracle_step.restype = ctypes.c_uint32
-        L.desloc_oracle_step.argtypes = [
-            ctypes.POINTER(OracleCfg), ctypes.c_int64, ctypes.c_double, ctypes.c_double,
-            ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
-            ctypes.c_void_p]
-        L.desloc_oracle_step_scaled.restype = ctypes.c_uint32
-        L.desloc_oracle_step_scaled.argtypes = L.desloc_oracle_step.argtypes + [ctypes.c_void_p]
-        L.desloc_oracle_norm_scales.restype = None
-        L.desloc_oracle_norm_scales.argtypes = [ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
-                                                ctypes.c_void_p, ctypes.c_double, ctypes.c_void_p,
-                                                ctypes.c_void_p]
-        L.desloc_oracle_worker_mean.restype = None
-        L.desloc_oracle_worker_mean.argtypes = [ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
-                                                ctypes.c_void_p, ctypes.c_void_p]
-        L.desloc_oracle_rel_change.restype = None
-        L.desloc_oracle_rel_change.argtypes = [ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
-                                               ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
-        L.desloc_oracle_run.restype = None
-        L.desloc_oracle_run.argtypes = [
-            ctypes.POINTER(OracleCfg), ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p,
-            ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p,
-            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
-        _lib = L
+        _lib = configure(ctypes.CDLL(build()))
     return _lib
 
 

@@ -29,6 +29,22 @@ def test_library_exports_every_declared_symbol(d):
         assert hasattr(L, n), f"{n} declared in desloc.h but not exported"
 
 
+def test_header_is_plain_c_and_a_c_program_links(d, tmp_path):
+    """include/desloc.h compiles as strict C99, and a C program linked against the shared
+    library can call the host-only entry points."""
+    import subprocess
+    from paper_2505_22549_b200 import binding
+    inc = os.path.join(ROOT, "include")
+    src = os.path.join(ROOT, "tests", "c_abi", "abi_check.c")
+    exe = str(tmp_path / "abi_check")
+    libdir = os.path.dirname(binding.LIB_PATH)
+    subprocess.check_call(["gcc", "-std=c99", "-pedantic", "-Wall", "-Wextra", "-Werror", "-I", inc,
+                           src, "-o", exe, "-L", libdir, "-ldesloc", f"-Wl,-rpath,{libdir}"])
+    r = subprocess.run([exe], capture_output=True, text=True)
+    assert r.returncode == 0, r.stdout + r.stderr
+    assert "abi_check: ok" in r.stdout
+
+
 def test_sync_mask_matches_oracle_schedule(d):
     for opt, oid in (("adam", oracle.ADAM), ("adopt", oracle.ADOPT), ("sgdm", oracle.SGDM)):
         for K in [(4, 8, 16), (1, 1, 1), (16, 64, 256), (0, 0, 0), (3, 0, 7), (256, 768, 1536)]:

@@ -567,3 +567,32 @@ def test_worker_mean_closed_forms_and_doubling_keeps_the_mean():
     mean = oracle.worker_mean(f32(base))
     doubled = f32(np.concatenate([base, np.tile(mean, (4, 1))]))
     assert np.array_equal(oracle.worker_mean(doubled), mean)
+
+
+# --------------------------------------------------------------------------- closed forms, one step
+def test_adam_stability_term_sits_inside_the_root():
+    """Algorithm 2: d = eta / sqrt(v + lambda^2) * u.  One step from zero states with g = 3,
+    beta1 = beta2 = 1/2, lambda = 4: u = 3/2, v = 9/2, x = x0 - eta * 1.5 / sqrt(4.5 + 16)."""
+    cfg = oracle.make_cfg(1, ADAM, beta1=0.5, beta2=0.5, eps=4.0, Kx=0, Ku=0, Kv=0)
+    x, u, v = f32([[1.0]]), zeros(1, 1), zeros(1, 1)
+    oracle.step(cfg, 0, 0.5, x, u, v, f32([[3.0]]))
+    assert float(u[0, 0]) == 1.5 and float(v[0, 0]) == 4.5
+    want = 1.0 - 0.5 * 1.5 / math.sqrt(4.5 + 16.0)
+    assert abs(float(x[0, 0]) - want) < 1e-7
+    assert abs(float(x[0, 0]) - (1.0 - 0.5 * 1.5 / (math.sqrt(4.5) + 4.0))) > 1e-2   # not sqrt(v) + lambda
+
+
+def test_adopt_normalised_gradient_clip_is_two_sided():
+    """Optional ADOPT clip: g / max(sqrt(v_prev), eps) is clamped to [-c, c].  With v_prev = 1/4,
+    g = (4, -4, 0.5): ratios (8, -8, 1) -> (2, -2, 1) for c = 2; m = (1 - beta1) * that."""
+    cfg = oracle.make_cfg(1, ADOPT, beta1=0.5, beta2=0.5, eps=1e-6, Kx=0, Ku=0, Kv=0,
+                          flags=oracle.FLAG_ADOPT_NORM_CLIP)
+    x, u, v = zeros(1, 3), zeros(1, 3), f32([[0.25, 0.25, 0.25]])
+    oracle.step(cfg, 0, 1.0, x, u, v, f32([[4.0, -4.0, 0.5]]), clip_bound=2.0)
+    assert np.array_equal(u[0], f32([1.0, -1.0, 0.5]))
+    assert np.array_equal(x[0], f32([-1.0, 1.0, -0.5]))
+    assert np.array_equal(v[0], f32([0.125 + 8.0, 0.125 + 8.0, 0.125 + 0.125]))
+    # c = 0 (the bound at step 0 of the t^(1/4) schedule) zeroes the direction, v still updates
+    x, u, v = zeros(1, 3), zeros(1, 3), zeros(1, 3)
+    oracle.step(cfg, 0, 1.0, x, u, v, f32([[4.0, -4.0, 0.5]]), clip_bound=0.0)
+    assert np.array_equal(u[0], f32([0.0, 0.0, 0.0])) and np.all(v[0] > 0)
