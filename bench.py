@@ -487,6 +487,10 @@ def main():
                     help="override the workload's worker count M (exploration only)")
     ap.add_argument("--post-average", action="store_true",
                     help="average after the update (ordering of Algorithms 4-5) instead of before")
+    ap.add_argument("--grad-dtype", default=None, choices=["f32", "bf16"],
+                    help="override the workload's gradient dtype (exploration only)")
+    ap.add_argument("--opt", default=None, choices=["adam", "adopt", "sgdm"],
+                    help="override the workload's optimizer (exploration only)")
     ap.add_argument("--skip-e2e", action="store_true", help="omit the host-buffer leg (profiling)")
     ap.add_argument("--skip-cpu", action="store_true", help="omit the CPU oracle leg (profiling)")
     args = ap.parse_args()
@@ -494,6 +498,11 @@ def main():
     w = di.WORKLOADS[args.workload]
     if args.workers:
         w = w.replace(name=f"{w.name}_M{args.workers}", M=args.workers)
+    if args.grad_dtype:
+        w = w.replace(name=f"{w.name}_{args.grad_dtype}", grad_dtype=args.grad_dtype)
+    if args.opt:
+        w = w.replace(name=f"{w.name}_{args.opt}", opt=args.opt,
+                      adopt_norm_clip=(args.opt == "adopt"))
     if args.impl == "reference":
         return run_reference(args, w)
     return run_ours(args, w)
