@@ -24,6 +24,16 @@
 #ifndef DESLOC_SPLIT_LARGE_M
 #define DESLOC_SPLIT_LARGE_M 1
 #endif
+// Cache policy of the state and gradient accesses (0 = .cs evict-first, 1 = default,
+// 2 = .cg / L2 only).  Measured on B200: plain loads with plain stores are 2 % faster than
+// evict-first on every workload (27.0 against 27.55 ms on 1.7 B x 4); changing only one side
+// gains nothing.
+#ifndef DESLOC_LD_MODE
+#define DESLOC_LD_MODE 1
+#endif
+#ifndef DESLOC_ST_MODE
+#define DESLOC_ST_MODE 1
+#endif
 // 1: hardware reciprocal square root (about 2 ulp) instead of IEEE sqrt + division in the Adam
 // direction and the ADOPT normaliser.
 #ifndef DESLOC_FAST_MATH
@@ -83,15 +93,37 @@ struct FV {
     float a[VEC];
 };
 
-// ---- global memory access: streaming (evict-first) 128-bit or scalar ---------------------
+// ---- global memory access: 128-bit or scalar, cache policy per DESLOC_LD/ST_MODE ----------
+template <typename T>
+__device__ __forceinline__ T ld_stream(const T *p) {
+#if DESLOC_LD_MODE == 0
+    return __ldcs(p);
+#elif DESLOC_LD_MODE == 1
+    return *p;
+#else
+    return __ldcg(p);
+#endif
+}
+
+template <typename T>
+__device__ __forceinline__ void st_stream(T *p, const T &v) {
+#if DESLOC_ST_MODE == 0
+    __stcs(p, v);
+#elif DESLOC_ST_MODE == 1
+    *p = v;
+#else
+    __stcg(p, v);
+#endif
+}
+
 template <int VEC>
 __device__ __forceinline__ FV<VEC> ld_f32(const char *base, long long elem) {
     FV<VEC> r;
     if constexpr (VEC == 4) {
-        const float4 t = __ldcs(reinterpret_cast<const float4 *>(base) + (elem >> 2));
+        const float4 t = ld_stream(reinterpret_cast<const float4 *>(base) + (elem >> 2));
         r.a[0] = t.x; r.a[1] = t.y; r.a[2] = t.z; r.a[3] = t.w;
     } else {
-        r.a[0] = __ldcs(reinterpret_cast<const float *>(base) + elem);
+        r.a[0] = ld_stream(reinterpret_cast<const float *>(base) + elem);
     }
     return r;
 }
@@ -99,10 +131,10 @@ __device__ __forceinline__ FV<VEC> ld_f32(const char *base, long long elem) {
 template <int VEC>
 __device__ __forceinline__ void st_f32(char *base, long long elem, const FV<VEC> &r) {
     if constexpr (VEC == 4) {
-        __stcs(reinterpret_cast<float4 *>(base) + (elem >> 2),
-               make_float4(r.a[0], r.a[1], r.a[2], r.a[3]));
+        st_stream(reinterpret_cast<float4 *>(base) + (elem >> 2),
+                  make_float4(r.a[0], r.a[1], r.a[2], r.a[3]));
     } else {
-        __stcs(reinterpret_cast<float *>(base) + elem, r.a[0]);
+        st_stream(reinterpret_cast<float *>(base) + elem, r.a[0]);
     }
 }
 
@@ -113,13 +145,13 @@ __device__ __forceinline__ FV<VEC> ld_grad(const char *base, long long elem) {
         r = ld_f32<VEC>(base, elem);
     } else if constexpr (VEC == 4) {
         // four bf16 in 8 bytes; bf16 -> fp32 is a 16-bit shift (exact)
-        const uint2 t = __ldcs(reinterpret_cast<const uint2 *>(base) + (elem >> 2));
+        const uint2 t = ld_stream(reinterpret_cast<const uint2 *>(base) + (elem >> 2));
         r.a[0] = __uint_as_float(t.x << 16);
         r.a[1] = __uint_as_float(t.x & 0xffff0000u);
         r.a[2] = __uint_as_float(t.y << 16);
         r.a[3] = __uint_as_float(t.y & 0xffff0000u);
     } else {
-        const unsigned short t = __ldcs(reinterpret_cast<const unsigned short *>(base) + elem);
+        const unsigned short t = ld_stream(reinterpret_cast<const unsigned short *>(base) + elem);
         r.a[0] = __uint_as_float(static_cast<unsigned>(t) << 16);
     }
     return r;
