@@ -39,6 +39,12 @@
 #ifndef DESLOC_FAST_MATH
 #define DESLOC_FAST_MATH 0
 #endif
+#ifndef DESLOC_BLOCK_THREADS
+#define DESLOC_BLOCK_THREADS 256
+#endif
+#ifndef DESLOC_MINB_SMALL_M
+#define DESLOC_MINB_SMALL_M 3
+#endif
 #ifndef DESLOC_MINB_LARGE_M
 #define DESLOC_MINB_LARGE_M 3
 #endif
@@ -47,8 +53,8 @@ namespace desloc {
 
 constexpr int OPT_ADAM = 0, OPT_ADOPT = 1, OPT_SGDM = 2;
 constexpr int SYNC_X = 1, SYNC_U = 2, SYNC_V = 4;
-constexpr int BLOCK_THREADS = 256;
-constexpr int CHUNK_ELEMS = 4096;  // 256 threads x 4 elements x 4 positions
+constexpr int BLOCK_THREADS = DESLOC_BLOCK_THREADS;
+constexpr int CHUNK_ELEMS = BLOCK_THREADS * 16;  // 256 threads x 4 elements x 4 rounds = 4096
 constexpr int MAX_MT = 8;          // largest worker count with a register-resident kernel
 
 struct __align__(16) Chunk {
@@ -437,7 +443,7 @@ __device__ __forceinline__ void process_chunk(const StepArgs &a, char *const (*s
 }
 
 template <int OPT, int MASK, int MT, typename GT, bool POST>
-__global__ void __launch_bounds__(BLOCK_THREADS, (MT <= 4 ? 3 : ((OPT == OPT_SGDM || POST) ? 2 : DESLOC_MINB_LARGE_M)))
+__global__ void __launch_bounds__(BLOCK_THREADS, (MT <= 4 ? DESLOC_MINB_SMALL_M : ((OPT == OPT_SGDM || POST) ? 2 : DESLOC_MINB_LARGE_M)))
 desloc_step_kernel(const __grid_constant__ StepArgs a) {
     __shared__ char *sp[4][MT];
     __shared__ float sscale[MT];

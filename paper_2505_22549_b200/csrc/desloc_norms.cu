@@ -81,7 +81,7 @@ __device__ __forceinline__ float sumsq8_bf16(const uint4 &t, float acc) {
 }
 
 template <typename GT>
-__global__ void __launch_bounds__(BLOCK_THREADS, 8)
+__global__ void __launch_bounds__(BLOCK_THREADS, 3)
 sumsq_kernel(const Chunk *chunks, long long nchunks, const void *const *g, int nt, int M,
              float *partial) {
     __shared__ float warp_sums[BLOCK_THREADS / 32];
@@ -93,45 +93,48 @@ sumsq_kernel(const Chunk *chunks, long long nchunks, const void *const *g, int n
         const int m = static_cast<int>(item / ngroups);
         const long long c0 = q * SUMSQ_GROUP;
         float acc0 = 0.f, acc1 = 0.f;
-        // four chunks per iteration; full, 16-byte aligned bf16 chunks take the wide path with
-        // all eight 128-bit loads of the iteration issued before the first use
-#pragma unroll 1
-        for (int k = 0; k < SUMSQ_GROUP; k += 4) {
-            if constexpr (sizeof(GT) == 2) {
+        if constexpr (sizeof(GT) == 2) {
+            // All chunk descriptors and gradient pointers of the group first (one dependent-load
+            // chain for the whole item), then the data: full, 16-byte aligned bf16 chunks take
+            // 128-bit loads, eight of them in flight per thread.
+            const uint4 *wide[SUMSQ_GROUP];
+#pragma unroll
+            for (int j = 0; j < SUMSQ_GROUP; ++j) {
+                wide[j] = nullptr;
+                if (c0 + j < nchunks) {
+                    const Chunk ch = chunks[c0 + j];
+                    const char *base =
+                        reinterpret_cast<const char *>(g[static_cast<long long>(m) * nt + ch.tensor]) +
+                        ch.start * 2;
+                    if (ch.count == CHUNK_ELEMS && (reinterpret_cast<uintptr_t>(base) & 15u) == 0)
+                        wide[j] = reinterpret_cast<const uint4 *>(base);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < SUMSQ_GROUP; k += 4) {
                 uint4 r[4][2];
-                bool wide[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    wide[j] = false;
-                    if (c0 + k + j < nchunks) {
-                        const Chunk ch = chunks[c0 + k + j];
-                        const char *base =
-                            reinterpret_cast<const char *>(g[static_cast<long long>(m) * nt + ch.tensor]) +
-                            ch.start * 2;
-                        wide[j] = ch.count == CHUNK_ELEMS && (reinterpret_cast<uintptr_t>(base) & 15u) == 0;
-                        if (wide[j]) {
-                            const uint4 *p = reinterpret_cast<const uint4 *>(base);
-                            r[j][0] = __ldcs(p + tid);
-                            r[j][1] = __ldcs(p + tid + BLOCK_THREADS);
-                        }
+                    if (wide[k + j]) {
+                        r[j][0] = ld_stream(wide[k + j] + tid);
+                        r[j][1] = ld_stream(wide[k + j] + tid + BLOCK_THREADS);
                     }
                 }
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    if (wide[j]) {
+                    if (wide[k + j]) {
                         acc0 = sumsq8_bf16(r[j][0], acc0);
                         acc1 = sumsq8_bf16(r[j][1], acc1);
                     } else if (c0 + k + j < nchunks) {
                         acc0 = chunk_sumsq<GT>(chunks[c0 + k + j], g, nt, m, acc0);
                     }
                 }
-            } else {
-#pragma unroll
-                for (int j = 0; j < 4; j += 2) {
-                    if (c0 + k + j < nchunks) acc0 = chunk_sumsq<GT>(chunks[c0 + k + j], g, nt, m, acc0);
-                    if (c0 + k + j + 1 < nchunks)
-                        acc1 = chunk_sumsq<GT>(chunks[c0 + k + j + 1], g, nt, m, acc1);
-                }
+            }
+        } else {
+#pragma unroll 1
+            for (int k = 0; k < SUMSQ_GROUP; k += 2) {
+                if (c0 + k < nchunks) acc0 = chunk_sumsq<GT>(chunks[c0 + k], g, nt, m, acc0);
+                if (c0 + k + 1 < nchunks) acc1 = chunk_sumsq<GT>(chunks[c0 + k + 1], g, nt, m, acc1);
             }
         }
         const float total = block_sum(acc0 + acc1, warp_sums);
