@@ -45,6 +45,9 @@
 #ifndef DESLOC_MINB_SMALL_M
 #define DESLOC_MINB_SMALL_M 3
 #endif
+#ifndef DESLOC_MINB_POST_LARGE_M
+#define DESLOC_MINB_POST_LARGE_M 2
+#endif
 #ifndef DESLOC_MINB_LARGE_M
 #define DESLOC_MINB_LARGE_M 3
 #endif
@@ -443,7 +446,7 @@ __device__ __forceinline__ void process_chunk(const StepArgs &a, char *const (*s
 }
 
 template <int OPT, int MASK, int MT, typename GT, bool POST>
-__global__ void __launch_bounds__(BLOCK_THREADS, (MT <= 4 ? DESLOC_MINB_SMALL_M : ((OPT == OPT_SGDM || POST) ? 2 : DESLOC_MINB_LARGE_M)))
+__global__ void __launch_bounds__(BLOCK_THREADS, (MT <= 4 ? DESLOC_MINB_SMALL_M : ((OPT == OPT_SGDM || POST) ? DESLOC_MINB_POST_LARGE_M : DESLOC_MINB_LARGE_M)))
 desloc_step_kernel(const __grid_constant__ StepArgs a) {
     __shared__ char *sp[4][MT];
     __shared__ float sscale[MT];
