@@ -281,13 +281,10 @@ def run_ours(args, w):
     total_ms = ev[0].elapsed_time(ev[-1])
     per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
     clocks = sampler.stop(wall0, wall1) if rank == 0 else None
-    if world > 1:
-        tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
-        lt = torch.tensor([launches], dtype=torch.int64, device=dev)
-        dist.all_reduce(lt, op=dist.ReduceOp.SUM)
-        launches = int(lt.item())
+    # every multi-GPU number is the slowest rank's; launches add up (helpers covered by the
+    # world-size-2 gloo tests)
+    total_ms = d.dist.max_over_ranks(total_ms, dev)
+    launches = d.dist.sum_over_ranks(launches, dev)
     value = world * w.M * w.N * args.steps / (total_ms * 1e-3) / 1e9
 
     # ---- per-mask timing (outside the headline region): local, x-only, all-sync ---------------
@@ -462,11 +459,8 @@ def run_e2e(args, w, eng, G, X, offs, dev, world, barrier):
     e1.record(stream)
     barrier()
     ms = e0.elapsed_time(e1)
-    if world > 1:
-        import torch.distributed as dist
-        tt = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms = float(tt.item())
+    import paper_2505_22549_b200 as d
+    ms = d.dist.max_over_ranks(ms, dev)
     return {"value": world * w.M * w.N * steps / (ms * 1e-3) / 1e9, "unit": UNIT,
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": last[1] * 4, "steps": steps,
             "ms_per_step": ms / steps,

@@ -573,11 +573,15 @@ int desloc_get_grad_norms(desloc_ctx *ctx, float *norms_out, float *scales_out, 
     if (!ctx) return DESLOC_E_NULL;
     const size_t bytes = static_cast<size_t>(ctx->cfg.M) * sizeof(float);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = cudaSuccess;
+    int dev_before = -1;
+    cudaError_t e = cudaGetDevice(&dev_before);
+    if (e == cudaSuccess && dev_before != ctx->device) e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
     if (norms_out) e = cudaMemcpyAsync(norms_out, ctx->res.d_norms, bytes, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess && scales_out)
         e = cudaMemcpyAsync(scales_out, ctx->res.d_norms + ctx->cfg.M, bytes, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (dev_before != ctx->device) cudaSetDevice(dev_before);
     return e == cudaSuccess ? DESLOC_OK : cuda_fail(ctx, e);
 }
 
@@ -635,7 +639,8 @@ int desloc_set_workers(desloc_ctx *ctx, int32_t M_new, int32_t first_new, float 
     if (e == cudaSuccess) {
         try {
             e = make_worker_res(fresh, M_new, nt, ctx->nchunks, has_v, x, u, v);
-            ctx->last_grads.assign(static_cast<size_t>(nptr_new), nullptr);
+            if (ctx->last_grads.capacity() < static_cast<size_t>(nptr_new))
+                ctx->last_grads.reserve(static_cast<size_t>(nptr_new));  // may throw; no state changed yet
         } catch (const std::bad_alloc &) {
             e = cudaErrorMemoryAllocation;
         }
@@ -658,6 +663,7 @@ int desloc_set_workers(desloc_ctx *ctx, int32_t M_new, int32_t first_new, float 
     if (e == cudaSuccess) {
         free_worker_res(ctx->res);
         ctx->res = fresh;
+        ctx->last_grads.assign(static_cast<size_t>(nptr_new), nullptr);  // capacity reserved above
         ctx->cfg.M = M_new;
         ctx->nptr = nptr_new;
         ctx->next_slot = 0;
