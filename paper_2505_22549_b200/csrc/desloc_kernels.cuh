@@ -24,6 +24,9 @@
 #ifndef DESLOC_SPLIT_LARGE_M
 #define DESLOC_SPLIT_LARGE_M 1
 #endif
+#ifndef DESLOC_SPLIT_LARGE_M_POST
+#define DESLOC_SPLIT_LARGE_M_POST 1
+#endif
 // Cache policy of the state and gradient accesses (0 = .cs evict-first, 1 = default,
 // 2 = .cg / L2 only).  Measured on B200: plain loads with plain stores are 2 % faster than
 // evict-first on every workload (27.0 against 27.55 ms on 1.7 B x 4); changing only one side
@@ -345,6 +348,81 @@ __device__ __forceinline__ void process_tile_split(const StepArgs &a, char *cons
     worker_batch<OPT, MASK, MT, GT, VEC, 4, MT - 4>(a, sp, sscale, e, xb, ub, vb);
 }
 
+// ---- post-average tile for many workers ---------------------------------------------------
+// Averages are taken over the UPDATED values, so every worker's new u, v must exist before any
+// parameter step.  Phase A updates the states four workers at a time and keeps them; phase B
+// forms the means of the synced ones; phase C loads x four workers at a time and steps it; a
+// synced x is averaged last.  Same arithmetic and summation tree as process_tile.
+template <int OPT, int MT, typename GT, int VEC, int M0, int B>
+__device__ __forceinline__ void post_states_batch(const StepArgs &a, char *const (*sp)[MT],
+                                                  const float *sscale, long long e,
+                                                  FV<VEC> (&UN)[MT], FV<VEC> (&VN)[MT]) {
+    FV<VEC> G[B], U[B], V[B];
+#pragma unroll
+    for (int b = 0; b < B; ++b) {
+        G[b] = ld_grad<VEC, GT>(sp[3][M0 + b], e);
+        U[b] = ld_f32<VEC>(sp[1][M0 + b], e);
+        if constexpr (OPT != OPT_SGDM) V[b] = ld_f32<VEC>(sp[2][M0 + b], e);
+    }
+#pragma unroll
+    for (int b = 0; b < B; ++b) {
+#pragma unroll
+        for (int c = 0; c < VEC; ++c) {
+            const float vown = OPT != OPT_SGDM ? V[b].a[c] : 0.f;
+            state_update<OPT>(a, G[b].a[c] * sscale[M0 + b], U[b].a[c], vown, vown,
+                              UN[M0 + b].a[c], VN[M0 + b].a[c]);
+        }
+    }
+}
+
+template <int OPT, int MASK, int MT, int VEC, int M0, int B>
+__device__ __forceinline__ void post_params_batch(const StepArgs &a, char *const (*sp)[MT],
+                                                  long long e, const FV<VEC> (&UN)[MT],
+                                                  const FV<VEC> (&VN)[MT], FV<VEC> (&XN)[MT]) {
+    FV<VEC> X[B];
+#pragma unroll
+    for (int b = 0; b < B; ++b) X[b] = ld_f32<VEC>(sp[0][M0 + b], e);
+#pragma unroll
+    for (int b = 0; b < B; ++b) {
+#pragma unroll
+        for (int c = 0; c < VEC; ++c)
+            XN[M0 + b].a[c] = param_step<OPT>(a, X[b].a[c], UN[M0 + b].a[c], VN[M0 + b].a[c]);
+        if constexpr (!(MASK & SYNC_X)) st_f32<VEC>(sp[0][M0 + b], e, XN[M0 + b]);
+        st_f32<VEC>(sp[1][M0 + b], e, UN[M0 + b]);
+        if constexpr (OPT != OPT_SGDM) st_f32<VEC>(sp[2][M0 + b], e, VN[M0 + b]);
+    }
+}
+
+template <int VEC, int MT>
+__device__ __forceinline__ void replace_by_mean(FV<VEC> (&S)[MT]) {
+#pragma unroll
+    for (int c = 0; c < VEC; ++c) {
+        float s[MT];
+#pragma unroll
+        for (int m = 0; m < MT; ++m) s[m] = S[m].a[c];
+        const float mean = mean_of<MT>(s);
+#pragma unroll
+        for (int m = 0; m < MT; ++m) S[m].a[c] = mean;
+    }
+}
+
+template <int OPT, int MASK, int MT, typename GT, int VEC>
+__device__ __forceinline__ void process_tile_split_post(const StepArgs &a, char *const (*sp)[MT],
+                                                        const float *sscale, long long e) {
+    FV<VEC> UN[MT], VN[MT], XN[MT];
+    post_states_batch<OPT, MT, GT, VEC, 0, 4>(a, sp, sscale, e, UN, VN);
+    post_states_batch<OPT, MT, GT, VEC, 4, MT - 4>(a, sp, sscale, e, UN, VN);
+    if constexpr (MASK & SYNC_U) replace_by_mean<VEC, MT>(UN);
+    if constexpr ((MASK & SYNC_V) && OPT != OPT_SGDM) replace_by_mean<VEC, MT>(VN);
+    post_params_batch<OPT, MASK, MT, VEC, 0, 4>(a, sp, e, UN, VN, XN);
+    post_params_batch<OPT, MASK, MT, VEC, 4, MT - 4>(a, sp, e, UN, VN, XN);
+    if constexpr (MASK & SYNC_X) {
+        replace_by_mean<VEC, MT>(XN);
+#pragma unroll
+        for (int m = 0; m < MT; ++m) st_f32<VEC>(sp[0][m], e, XN[m]);
+    }
+}
+
 // ---- one thread's tile: MT workers x UN positions of VEC elements ------------------------
 // sp[arr][m] are chunk-relative base pointers in shared memory (arr: 0 x, 1 u, 2 v, 3 g).
 // Position j covers elements e0 + j * pstride .. + VEC - 1; positions >= npos are skipped.
@@ -355,6 +433,13 @@ __device__ __forceinline__ void process_tile(const StepArgs &a, char *const (*sp
 #if DESLOC_SPLIT_LARGE_M
     if constexpr (!POST && MT > 4 && UN == 1 && OPT != OPT_SGDM) {
         if (FULL || npos > 0) process_tile_split<OPT, MASK, MT, GT, VEC>(a, sp, sscale, e0);
+        return;
+    }
+#endif
+#if DESLOC_SPLIT_LARGE_M_POST
+    // measured: faster for Adam (0.97-0.99 of copy bandwidth against 0.95), slower for ADOPT
+    if constexpr (POST && MT > 4 && UN == 1 && MASK != 0 && OPT == OPT_ADAM) {
+        if (FULL || npos > 0) process_tile_split_post<OPT, MASK, MT, GT, VEC>(a, sp, sscale, e0);
         return;
     }
 #endif
