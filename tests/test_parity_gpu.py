@@ -396,6 +396,47 @@ def test_two_contexts_on_two_streams_and_stream_changes():
     ea.close(); eb.close()
 
 
+def test_steps_allocate_no_device_memory():
+    """Everything a context needs is allocated by desloc_create(): free device memory (as the
+    driver reports it, which also sees allocations made outside torch) is the same before and
+    after many steps of every kind, with gradient pointers changing from step to step."""
+    d = _lib()
+    w = di.mini(di.WORKLOADS["cfg3_adopt_360m"], T=30).replace(K=(2, 3, 4))
+    dev = torch.device("cuda:0")
+    st = State(w, dev)
+    eng = make_engine(d, w, st)
+    alt = [b.clone() for b in st.g]
+    hflat = [torch.empty(st.nflat, dtype=st.g[0].dtype).pin_memory() for _ in range(w.M)]
+    hview = [[h[o:o + n] for o, n in zip(st.offs, w.numel)] for h in hflat]
+    st.fill_grads(0)
+    for kind in range(4):                       # first use of every entry point, then measure
+        eng.step(kind, 1e-3, st.views(st.g), clip_bound=1.0)
+    eng.step_normclip(4, 1e-3, st.views(alt), 0.5, clip_bound=1.0)
+    eng.step_host(5, 1e-3, hview, st.views(st.g), clip_bound=1.0)
+    cfg = d.make_config(w.M, w.numel, w.opt, w.grad_dtype, w.beta1, w.beta2, w.eps, 0.0, w.clip_rho,
+                        2, 3, 4, d.DESLOC_FLAG_ADOPT_NORM_CLIP)
+    flat = lambda bufs: [t.data_ptr() for lst in st.views(bufs) for t in lst]
+    d.desloc_step_static(cfg, flat(st.x), flat(st.u), flat(st.v), flat(st.g), 6, 1e-3, 1.0, 0,
+                         torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for t in range(7, 30):
+        gsel = st.g if t % 2 else alt
+        if t % 5 == 0:
+            eng.step_normclip(t, 1e-3, st.views(gsel), 0.5, clip_bound=1.0)
+        elif t % 7 == 0:
+            eng.step_host(t, 1e-3, hview, st.views(st.g), clip_bound=1.0)
+        elif t % 11 == 0:
+            d.desloc_step_static(cfg, flat(st.x), flat(st.u), flat(st.v), flat(gsel), t, 1e-3, 1.0, 0,
+                                 torch.cuda.current_stream().cuda_stream)
+        else:
+            eng.step(t, 1e-3, st.views(gsel), clip_bound=1.0)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
+    eng.close()
+
+
 def test_errors_are_status_codes_and_context_survives():
     d = _lib()
     dev = torch.device("cuda:0")
