@@ -55,18 +55,41 @@ __device__ __forceinline__ FV<VEC> ld_plain(const char *base, long long e) {
     return r;
 }
 
-template <int OPT, typename GT, bool POST, int VEC>
-__device__ __forceinline__ void generic_position(const StepArgs &a, const Chunk &ch, int mask,
+// CMASK >= 0: the sync mask is a compile-time constant (pre-average instantiations, so that
+// arrays that are not averaged cost no registers); CMASK < 0: taken from mask_rt.
+template <int OPT, typename GT, bool POST, int CMASK, int VEC>
+__device__ __forceinline__ void generic_position(const StepArgs &a, const Chunk &ch, int mask_rt,
                                                  long long e) {
+    const int mask = CMASK >= 0 ? CMASK : mask_rt;
     const int M = a.M;
     const bool sx = mask & SYNC_X, su = mask & SYNC_U, sv = (OPT != OPT_SGDM) && (mask & SYNC_V);
     if constexpr (!POST) {
         double ax[VEC] = {}, au[VEC] = {}, av[VEC] = {};
-        for (int m = 0; m < M; ++m) {
-            const Ptrs p = worker_ptrs<OPT, GT>(a, ch, m);
-            if (sx) acc_add<VEC>(ax, ld_plain<VEC>(p.x, e));
-            if (su) acc_add<VEC>(au, ld_plain<VEC>(p.u, e));
-            if (sv) acc_add<VEC>(av, ld_plain<VEC>(p.v, e));
+        // several workers at a time so that their pointer and data loads overlap (four when one
+        // array is averaged, two for two, one for three: more would spill under the register
+        // cap); the sums still run in the order m = 0..M-1
+        constexpr int NSYNC = CMASK < 0 ? 3 : ((CMASK & 1) + ((CMASK >> 1) & 1) + ((CMASK >> 2) & 1));
+        constexpr int NB = NSYNC <= 1 ? 4 : (NSYNC == 2 ? 2 : 1);
+#pragma unroll 1
+        for (int m0 = 0; m0 < M; m0 += NB) {
+            FV<VEC> bx[NB], bu[NB], bv[NB];
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                if (m0 + j < M) {
+                    const Ptrs p = worker_ptrs<OPT, GT>(a, ch, m0 + j);
+                    if (sx) bx[j] = ld_plain<VEC>(p.x, e);
+                    if (su) bu[j] = ld_plain<VEC>(p.u, e);
+                    if (sv) bv[j] = ld_plain<VEC>(p.v, e);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                if (m0 + j < M) {
+                    if (sx) acc_add<VEC>(ax, bx[j]);
+                    if (su) acc_add<VEC>(au, bu[j]);
+                    if (sv) acc_add<VEC>(av, bv[j]);
+                }
+            }
         }
         const FV<VEC> xb = acc_mean<VEC>(ax, M), ub = acc_mean<VEC>(au, M), vb = acc_mean<VEC>(av, M);
         for (int m = 0; m < M; ++m) {
@@ -178,7 +201,7 @@ __device__ __forceinline__ void generic_position(const StepArgs &a, const Chunk 
     }
 }
 
-template <int OPT, typename GT, bool POST>
+template <int OPT, typename GT, bool POST, int CMASK>
 __global__ void __launch_bounds__(BLOCK_THREADS, 4)
 desloc_step_generic_kernel(const __grid_constant__ StepArgs a, const int mask) {
     __shared__ int s_mis;
@@ -202,26 +225,46 @@ desloc_step_generic_kernel(const __grid_constant__ StepArgs a, const int mask) {
         if (!scalar_path) {
             const int n4 = ch.count >> 2;
             for (int p0 = tid; p0 < n4; p0 += BLOCK_THREADS)
-                generic_position<OPT, GT, POST, 4>(a, ch, mask, static_cast<long long>(p0) * 4);
+                generic_position<OPT, GT, POST, CMASK, 4>(a, ch, mask, static_cast<long long>(p0) * 4);
             const int rem = ch.count & 3;
-            if (tid < rem) generic_position<OPT, GT, POST, 1>(a, ch, mask, (n4 << 2) + tid);
+            if (tid < rem) generic_position<OPT, GT, POST, CMASK, 1>(a, ch, mask, (n4 << 2) + tid);
         } else {
             for (int e = tid; e < ch.count; e += BLOCK_THREADS)
-                generic_position<OPT, GT, POST, 1>(a, ch, mask, e);
+                generic_position<OPT, GT, POST, CMASK, 1>(a, ch, mask, e);
         }
     }
 }
 
-template <int OPT, bool POST>
-static const void *pick_generic(bool bf16) {
-    return bf16 ? reinterpret_cast<const void *>(&desloc_step_generic_kernel<OPT, bf16_t, POST>)
-                : reinterpret_cast<const void *>(&desloc_step_generic_kernel<OPT, float, POST>);
+template <int OPT, typename GT, bool POST, int CMASK>
+static const void *generic_ptr() {
+    return reinterpret_cast<const void *>(&desloc_step_generic_kernel<OPT, GT, POST, CMASK>);
 }
 
-const void *lookup_generic_kernel(int opt, bool post, bool bf16) {
-    if (opt == OPT_ADAM) return post ? pick_generic<OPT_ADAM, true>(bf16) : pick_generic<OPT_ADAM, false>(bf16);
-    if (opt == OPT_ADOPT) return post ? pick_generic<OPT_ADOPT, true>(bf16) : pick_generic<OPT_ADOPT, false>(bf16);
-    if (opt == OPT_SGDM) return post ? pick_generic<OPT_SGDM, true>(bf16) : pick_generic<OPT_SGDM, false>(bf16);
+template <int OPT, typename GT>
+static const void *pick_generic(bool post, int mask) {
+    if (post) return generic_ptr<OPT, GT, true, -1>();
+    switch (mask) {
+        case 1: return generic_ptr<OPT, GT, false, 1>();
+        case 2: return generic_ptr<OPT, GT, false, 2>();
+        case 3: return generic_ptr<OPT, GT, false, 3>();
+        default: break;
+    }
+    if constexpr (OPT != OPT_SGDM) {
+        switch (mask) {
+            case 4: return generic_ptr<OPT, GT, false, 4>();
+            case 5: return generic_ptr<OPT, GT, false, 5>();
+            case 6: return generic_ptr<OPT, GT, false, 6>();
+            case 7: return generic_ptr<OPT, GT, false, 7>();
+            default: break;
+        }
+    }
+    return nullptr;
+}
+
+const void *lookup_generic_kernel(int opt, bool post, bool bf16, int mask) {
+    if (opt == OPT_ADAM) return bf16 ? pick_generic<OPT_ADAM, bf16_t>(post, mask) : pick_generic<OPT_ADAM, float>(post, mask);
+    if (opt == OPT_ADOPT) return bf16 ? pick_generic<OPT_ADOPT, bf16_t>(post, mask) : pick_generic<OPT_ADOPT, float>(post, mask);
+    if (opt == OPT_SGDM) return bf16 ? pick_generic<OPT_SGDM, bf16_t>(post, mask) : pick_generic<OPT_SGDM, float>(post, mask);
     return nullptr;
 }
 

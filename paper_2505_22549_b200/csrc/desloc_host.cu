@@ -280,7 +280,8 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
         const bool per_worker_items = (c.M == 1) || (kmask == 0 && c.M > desloc::MAX_MT);
         const bool generic = kmask != 0 && c.M > desloc::MAX_MT;
         const void *fn = generic
-                             ? desloc::lookup_generic_kernel(c.opt, post, c.grad_dtype == DESLOC_BF16)
+                             ? desloc::lookup_generic_kernel(c.opt, post, c.grad_dtype == DESLOC_BF16,
+                                                             static_cast<int>(kmask))
                              : desloc::lookup_step_kernel(c.opt, post, c.grad_dtype == DESLOC_BF16,
                                                           c.M, static_cast<int>(kmask));
         if (!fn) {

@@ -636,6 +636,6 @@ desloc_local_kernel(const __grid_constant__ StepArgs a) {
 const void *lookup_step_kernel(int opt, bool post, bool bf16, int mt, int mask);
 
 // Runtime-M kernel for sync steps of M > MAX_MT; launched with (StepArgs, int mask).
-const void *lookup_generic_kernel(int opt, bool post, bool bf16);
+const void *lookup_generic_kernel(int opt, bool post, bool bf16, int mask);
 
 }  // namespace desloc
