@@ -379,6 +379,8 @@ def run_ours(args, w):
     if rank == 0:
         cpu = (time_oracle(w, seconds_target=15.0) if not args.skip_cpu else
                {"value": None, "unit": UNIT, "cores": 0, "kind": "oracle", "sample": "skipped"})
+        if not args.skip_cpu:   # the same routine on one core, for the per-core figure
+            cpu["single_thread"] = time_oracle(w, seconds_target=4.0, threads=1)["value"]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps,
@@ -393,7 +395,8 @@ def run_ours(args, w):
                        "ordering": "post-average" if args.post_average else "pre-average",
                        "masks_in_timed_region": masks},
             "roofline": roofline, "by_mask": by_mask, "normclip_step": normclip, "graph_window": graph_info, "cpu_baseline": {k: cpu[k] for k in
-                                                                       ("value", "unit", "cores", "kind", "sample")},
+                                                                       ("value", "unit", "cores", "kind", "sample",
+                                                                        "single_thread") if k in cpu},
             "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
         }
         print(json.dumps(line), flush=True)
