@@ -180,6 +180,19 @@ def test_mini_workloads_full_oracle(name):
     print(name, worst)
 
 
+@pytest.mark.parametrize("name", ["cfg2_adam_135m", "cfg3_adopt_360m", "cfg5_adam_desloc",
+                                  "cfg5_sgdm_desloc"])
+def test_mini_workloads_full_horizon_and_periods(name):
+    """The workloads' own step counts (T = 256 / 512) and periods (up to K_v = 256) on the mini
+    model: the error bar must hold after the whole horizon, not only after a few steps."""
+    w = di.mini(di.WORKLOADS[name])
+    res = run_both(w, w.T)
+    worst = check(res)
+    want = [-(-w.T // k) for k in w.K[:2]] + ([-(-w.T // w.K[2])] if w.opt != "sgdm" else [0])
+    assert res["counters"] == [w.T] + want
+    print(name, w.T, worst)
+
+
 def test_persistent_grid_gives_identical_bits():
     w = di.mini(di.WORKLOADS["cfg2_adam_135m"], T=12).replace(K=(2, 3, 4))
     a = run_both(w, w.T, ctas_per_sm=0)
