@@ -93,10 +93,12 @@ sumsq_kernel(const Chunk *chunks, long long nchunks, const void *const *g, int n
         const int m = static_cast<int>(item / ngroups);
         const long long c0 = q * SUMSQ_GROUP;
         float acc0 = 0.f, acc1 = 0.f;
-        if constexpr (sizeof(GT) == 2) {
+        {
             // All chunk descriptors and gradient pointers of the group first (one dependent-load
-            // chain for the whole item), then the data: full, 16-byte aligned bf16 chunks take
-            // 128-bit loads, eight of them in flight per thread.
+            // chain for the whole item), then the data: full, 16-byte aligned chunks take 128-bit
+            // loads, eight of them in flight per thread (four bf16 chunks or two fp32 chunks).
+            constexpr int LPC = sizeof(GT) == 2 ? 2 : 4;  // 128-bit loads per thread and chunk
+            constexpr int CB = 8 / LPC;                   // chunks per batch
             const uint4 *wide[SUMSQ_GROUP];
 #pragma unroll
             for (int j = 0; j < SUMSQ_GROUP; ++j) {
@@ -105,36 +107,41 @@ sumsq_kernel(const Chunk *chunks, long long nchunks, const void *const *g, int n
                     const Chunk ch = chunks[c0 + j];
                     const char *base =
                         reinterpret_cast<const char *>(g[static_cast<long long>(m) * nt + ch.tensor]) +
-                        ch.start * 2;
+                        ch.start * static_cast<long long>(sizeof(GT));
                     if (ch.count == CHUNK_ELEMS && (reinterpret_cast<uintptr_t>(base) & 15u) == 0)
                         wide[j] = reinterpret_cast<const uint4 *>(base);
                 }
             }
 #pragma unroll
-            for (int k = 0; k < SUMSQ_GROUP; k += 4) {
-                uint4 r[4][2];
+            for (int k = 0; k < SUMSQ_GROUP; k += CB) {
+                uint4 r[CB][LPC];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < CB; ++j) {
                     if (wide[k + j]) {
-                        r[j][0] = ld_stream(wide[k + j] + tid);
-                        r[j][1] = ld_stream(wide[k + j] + tid + BLOCK_THREADS);
+#pragma unroll
+                        for (int l = 0; l < LPC; ++l)
+                            r[j][l] = ld_stream(wide[k + j] + tid + l * BLOCK_THREADS);
                     }
                 }
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < CB; ++j) {
                     if (wide[k + j]) {
-                        acc0 = sumsq8_bf16(r[j][0], acc0);
-                        acc1 = sumsq8_bf16(r[j][1], acc1);
+#pragma unroll
+                        for (int l = 0; l < LPC; ++l) {
+                            float &acc = (l & 1) ? acc1 : acc0;
+                            if constexpr (sizeof(GT) == 2) {
+                                acc = sumsq8_bf16(r[j][l], acc);
+                            } else {
+                                const float f[4] = {__uint_as_float(r[j][l].x), __uint_as_float(r[j][l].y),
+                                                    __uint_as_float(r[j][l].z), __uint_as_float(r[j][l].w)};
+#pragma unroll
+                                for (int q4 = 0; q4 < 4; ++q4) acc = fmaf(f[q4], f[q4], acc);
+                            }
+                        }
                     } else if (c0 + k + j < nchunks) {
                         acc0 = chunk_sumsq<GT>(chunks[c0 + k + j], g, nt, m, acc0);
                     }
                 }
-            }
-        } else {
-#pragma unroll 1
-            for (int k = 0; k < SUMSQ_GROUP; k += 2) {
-                if (c0 + k < nchunks) acc0 = chunk_sumsq<GT>(chunks[c0 + k], g, nt, m, acc0);
-                if (c0 + k + 1 < nchunks) acc1 = chunk_sumsq<GT>(chunks[c0 + k + 1], g, nt, m, acc1);
             }
         }
         const float total = block_sum(acc0 + acc1, warp_sums);

@@ -62,6 +62,35 @@ def test_normclip_step_matches_oracle(name, M, align):
     eng.close()
 
 
+@pytest.mark.parametrize("M", [2, 8])
+def test_normclip_with_fp32_gradients(M):
+    """fp32 gradients take their own wide path in the sum-of-squares kernel: full chunks, ragged
+    tails and misaligned tensors."""
+    import paper_2505_22549_b200 as d
+    numel = (4096 * 3, 4096 * 9 + 5, 17, 4096 * 8, 1000)
+    w = di.Workload("nc_f32", "adam", M, numel, "f32", "normal1", lr=1e-2, K=(2, 3, 4), seed=21)
+    dev = torch.device("cuda:0")
+    for align in (4, 1):
+        st = State(w, dev, align=align)
+        eng = make_engine(d, w, st)
+        ox, ou, ov = st.to_numpy(st.x), st.to_numpy(st.u), st.to_numpy(st.v)
+        valid = _valid(st)
+        for t in range(6):
+            st.fill_grads(t)
+            mx = f32r([50.0, 1e9, 5.0][t % 3])          # norm is about sqrt(N) = 290
+            g_host = st.to_numpy(st.g)
+            norms, scales = oracle.norm_scales(np.ascontiguousarray(g_host[:, valid]), mx)
+            eng.step_normclip(t, f32r(w.lr), st.views(st.g), mx)
+            got_n, got_s = eng.grad_norms()
+            assert np.allclose(got_n, norms, rtol=2e-6) and np.allclose(got_s, scales, rtol=2e-6)
+            oracle.step(oracle_cfg(w), t, f32r(w.lr), ox, ou, ov, g_host,
+                        gscale=np.asarray(got_s, dtype=np.float64))
+        torch.cuda.synchronize()
+        compare_per_tensor(st, st.to_numpy(st.x), ox, "x")
+        compare_per_tensor(st, st.to_numpy(st.v), ov, "v")
+        eng.close()
+
+
 def test_normclip_end_to_end_against_oracle_factors():
     """Same run but the oracle uses its own fp64 factors: the end state still meets the bar."""
     import paper_2505_22549_b200 as d
