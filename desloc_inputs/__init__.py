@@ -158,13 +158,18 @@ def fill_grads_(w: Workload, t: int, m: int, out: torch.Tensor, align: int = 1,
                 identical_workers: bool = False) -> None:
     """Write worker m's step-t gradient into the flat buffer `out` (fp32 or bf16).
 
-    normal1        N(0, 1)
+    normal1        N(0, 1) from host_normals(): the same bits on every host and library version
     normal_offset  N(0, sd 1e-3) plus one constant per (worker, tensor) drawn N(0, sd 1e-4)
     student_t3     1e-3 * z / sqrt((z1^2 + z2^2 + z3^2) / 3)
     With identical_workers every worker receives worker 0's stream.
     """
     dev = out.device
     mm = 0 if identical_workers else m
+    if w.grad_kind == "normal1":
+        # the small fp32 workloads draw from the generator defined in this module, on the host
+        z = host_normals(out.numel(), w.seed, 0x6AAD, t, mm).astype(np.float32)
+        out.copy_(torch.from_numpy(z).to(out.dtype))
+        return
     gen = torch.Generator(device=dev)
     gen.manual_seed(_mix(w.seed, 0x6AAD, t, mm))
     n = out.numel()
@@ -199,6 +204,38 @@ def fill_grads_(w: Workload, t: int, m: int, out: torch.Tensor, align: int = 1,
             raise ValueError(w.grad_kind)
         out[s:e].copy_(z)
         del z
+
+
+def host_normals(n: int, *key: int) -> np.ndarray:
+    """n standard normals in fp64 from a generator defined entirely here (independent of any
+    library's random stream): splitmix64 of (key, counter) -> two 53-bit uniforms -> Box-Muller.
+    The same key always gives the same bits on every host."""
+    base = np.uint64(_mix(0xB0C5, *key))
+    pairs = (n + 1) // 2
+    with np.errstate(over="ignore"):
+        ctr = base + np.arange(2 * pairs, dtype=np.uint64) * np.uint64(0x9E3779B97F4A7C15)
+        z = ctr
+        z = (z ^ (z >> np.uint64(30))) * np.uint64(0xBF58476D1CE4E5B9)
+        z = (z ^ (z >> np.uint64(27))) * np.uint64(0x94D049BB133111EB)
+        z = z ^ (z >> np.uint64(31))
+    unit = (z >> np.uint64(11)).astype(np.float64) * (1.0 / (1 << 53))
+    u1 = 1.0 - unit[0::2]            # (0, 1]: the logarithm stays finite
+    u2 = unit[1::2]
+    r = np.sqrt(-2.0 * np.log(u1))
+    out = np.empty(2 * pairs, dtype=np.float64)
+    out[0::2] = r * np.cos(2.0 * np.pi * u2)
+    out[1::2] = r * np.sin(2.0 * np.pi * u2)
+    return out[:n]
+
+
+def toy_rosenbrock_grads(x: np.ndarray, t: int, sigma: float = 1.5, seed: int = 0) -> np.ndarray:
+    """Noisy gradients of the toy problem f = (1 - x1)^2 + 100 (x2 - x1^2)^2 at the iterates
+    x [M, 2] (fp32): the exact gradient in fp64 plus sigma * N(0, 1) per worker and coordinate,
+    rounded to fp32.  A workload recipe: none of the optimizer's arithmetic is in here."""
+    x1, x2 = x[:, 0].astype(np.float64), x[:, 1].astype(np.float64)
+    g = np.stack([-2.0 * (1.0 - x1) - 400.0 * x1 * (x2 - x1 * x1), 200.0 * (x2 - x1 * x1)], axis=1)
+    noise = host_normals(g.size, seed, 0x7070, t).reshape(g.shape)
+    return np.ascontiguousarray(g + sigma * noise, dtype=np.float32)
 
 
 def sample_indices(numel: Sequence[int], n_hashed: int, seed: int = 0, edge: int = 64,

@@ -68,6 +68,12 @@ def configure(L: ctypes.CDLL) -> ctypes.CDLL:
         ctypes.c_void_p]
     L.desloc_oracle_step_scaled.restype = ctypes.c_uint32
     L.desloc_oracle_step_scaled.argtypes = L.desloc_oracle_step.argtypes + [ctypes.c_void_p]
+    L.desloc_oracle_step_full.restype = ctypes.c_uint32
+    L.desloc_oracle_step_full.argtypes = L.desloc_oracle_step_scaled.argtypes + [ctypes.c_void_p]
+    L.desloc_oracle_tensor_norms.restype = None
+    L.desloc_oracle_tensor_norms.argtypes = [ctypes.c_int32, ctypes.c_int64, ctypes.c_int32,
+                                             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                             ctypes.c_void_p, ctypes.c_void_p]
     L.desloc_oracle_norm_scales.restype = None
     L.desloc_oracle_norm_scales.argtypes = [ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
                                             ctypes.c_void_p, ctypes.c_double, ctypes.c_void_p,
@@ -143,22 +149,47 @@ def rel_change(now, then):
     return out
 
 
+def tensor_norms(a, offs, numel):
+    """L2 norms per (worker, tensor) and per worker of an [M, n] array (any float dtype, widened
+    to fp64 exactly); tensor k is a[:, offs[k] : offs[k] + numel[k]].  Returns ([M, nt], [M])."""
+    a64 = np.ascontiguousarray(a, dtype=np.float64)
+    if a64.ndim != 2:
+        raise ValueError("a must have shape [M, n]")
+    M, n = a64.shape
+    o = np.ascontiguousarray(offs, dtype=np.int64)
+    c = np.ascontiguousarray(numel, dtype=np.int64)
+    if o.shape != c.shape or o.ndim != 1 or np.any(o < 0) or np.any(o + c > n):
+        raise ValueError("offs / numel do not fit the array")
+    out = np.zeros((M, len(o)), dtype=np.float64)
+    tot = np.zeros(M, dtype=np.float64)
+    lib().desloc_oracle_tensor_norms(M, n, len(o), o.ctypes.data, c.ctypes.data, a64.ctypes.data,
+                                     out.ctypes.data, tot.ctypes.data)
+    return out, tot
+
+
 def step(cfg: OracleCfg, t: int, lr: float, x, u, v, g, clip_bound: float = 0.0,
-         gscale=None) -> int:
+         gscale=None, d_out=None) -> int:
     """One step in place on float32 arrays of shape [M, n]; returns the sync mask.
-    gscale: optional per-worker factors applied to g before the coordinate clip."""
+    gscale: optional per-worker factors applied to g before the coordinate clip.
+    d_out: optional float64 array [M, n] that receives every worker's update d_t."""
     M = cfg.M
     px, pu, pg = _check(x, M, "x"), _check(u, M, "u"), _check(g, M, "g")
     pv = _check(v, M, "v", allow_none=(cfg.opt == SGDM))
     n = x.shape[1]
     if u.shape != x.shape or g.shape != x.shape or (v is not None and v.shape != x.shape):
         raise ValueError("x, u, v, g must share one shape")
-    if gscale is not None:
-        gs = np.ascontiguousarray(gscale, dtype=np.float64)
-        assert gs.shape == (M,)
-        return int(lib().desloc_oracle_step_scaled(ctypes.byref(cfg), int(t), float(lr),
-                                                   float(clip_bound), n, n, px, pu, pv, pg,
-                                                   gs.ctypes.data))
+    if gscale is not None or d_out is not None:
+        gs = None
+        if gscale is not None:
+            gs = np.ascontiguousarray(gscale, dtype=np.float64)
+            assert gs.shape == (M,)
+        if d_out is not None and not (isinstance(d_out, np.ndarray) and d_out.dtype == np.float64
+                                      and d_out.shape == x.shape and d_out.flags["C_CONTIGUOUS"]):
+            raise ValueError("d_out must be a C-contiguous float64 array shaped like x")
+        return int(lib().desloc_oracle_step_full(
+            ctypes.byref(cfg), int(t), float(lr), float(clip_bound), n, n, px, pu, pv, pg,
+            gs.ctypes.data if gs is not None else None,
+            d_out.ctypes.data if d_out is not None else None))
     return int(lib().desloc_oracle_step(ctypes.byref(cfg), int(t), float(lr), float(clip_bound),
                                         n, n, px, pu, pv, pg))
 

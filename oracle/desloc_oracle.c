@@ -39,12 +39,19 @@
  *     algorithm listings) scales each worker's whole gradient by min(1, rho_norm/||g||_2)
  *     BEFORE the coordinate clip; no epsilon is added to the norm.
  *
+ *   - norms reported as diagnostics: the gradient norm is taken over the gradient as it is
+ *     read (before any clipping), the parameter norm over x_{t+1} as stored, the update norm
+ *     over d_t; each per worker and per tensor.
+ *
  * Pins (tests/test_oracle_pins.py): M=1 against torch.optim.Adam / AdamW / SGD
  * in fp64; identical gradients keep replicas equal to the single-worker run;
  * the worker-mean of u, v (and of x for SGDM) does not depend on the schedule;
  * three hand-worked examples in exact rationals; the clipping bounds of
  * Eqs. 5-6; the printed communication ratios (170x, 85x, 256x, 2x); full
- * agreement of the workers' inputs at multiples of lcm(K_x,K_u,K_v).
+ * agreement of the workers' inputs at multiples of lcm(K_x,K_u,K_v); d_t against
+ * the hand examples (both as eta u / sqrt(v) and as the difference of consecutive x), against
+ * the parameter change torch.optim makes at M = 1, and one-step closed forms; tensor norms
+ * against 3-4-5 style closed forms and numpy.linalg.norm.
  * Parity unpinned: the ADOPT normalised-gradient clip bound and the
  * weight-decay form are readings, not facts the paper fixes; the ADOPT rule
  * itself is pinned only by the hand example and brute force (no library has it).
@@ -101,10 +108,14 @@ static double worker_mean(const float *s, int64_t stride, int64_t i, int M) {
  * One DES-LOC step over n coordinates.  x, u, v, g are [M][stride] arrays
  * (worker-major), g already widened to fp32 (bf16 widens exactly).  v may be
  * NULL for SGDM.  Updates x, u, v in place; returns the sync mask used.
+ * gscale (may be NULL): per-worker factors applied to g before the coordinate clip.
+ * d_out (may be NULL): [M][stride] doubles, receives every worker's update d_t -- the quantity
+ * Algorithm 2 names d_t = eta_t u_t / sqrt(v_t + lambda^2) (eta_t u_t for ADOPT and SGDM),
+ * i.e. the step taken from the (possibly averaged) base, without the weight-decay term.
  */
-uint32_t desloc_oracle_step_scaled(const desloc_oracle_cfg *c, int64_t t, double lr,
-                                   double clip_bound, int64_t n, int64_t stride, float *x, float *u,
-                                   float *v, const float *g, const double *gscale) {
+uint32_t desloc_oracle_step_full(const desloc_oracle_cfg *c, int64_t t, double lr,
+                                 double clip_bound, int64_t n, int64_t stride, float *x, float *u,
+                                 float *v, const float *g, const double *gscale, double *d_out) {
     const int M = c->M;
     const uint32_t mask = desloc_oracle_sync_mask(c->opt, c->Kx, c->Ku, c->Kv, t);
     const int post = (c->flags & DESLOC_ORACLE_POST_AVERAGE) != 0;
@@ -181,6 +192,7 @@ uint32_t desloc_oracle_step_scaled(const desloc_oracle_cfg *c, int64_t t, double
             else
                 d = lr * un[m]; /* Algorithm 3 / SGDM */
             xn[m] = xp * (1.0 - lr * c->weight_decay) - d;
+            if (d_out) d_out[k] = d; /* the update d_t of Algorithms 2-3, kept in fp64 */
         }
         if (post && (mask & ORACLE_SYNC_X)) {
             double acc = 0.0;
@@ -199,6 +211,13 @@ uint32_t desloc_oracle_step_scaled(const desloc_oracle_cfg *c, int64_t t, double
     free(un);
     free(vn);
     return mask;
+}
+
+/* The same step with per-worker gradient factors (norm-based clipping) and no report of d. */
+uint32_t desloc_oracle_step_scaled(const desloc_oracle_cfg *c, int64_t t, double lr,
+                                   double clip_bound, int64_t n, int64_t stride, float *x, float *u,
+                                   float *v, const float *g, const double *gscale) {
+    return desloc_oracle_step_full(c, t, lr, clip_bound, n, stride, x, u, v, g, gscale, NULL);
 }
 
 uint32_t desloc_oracle_step(const desloc_oracle_cfg *c, int64_t t, double lr, double clip_bound,
@@ -251,6 +270,32 @@ void desloc_oracle_rel_change(int32_t M, int64_t n, int64_t stride, const float 
             den += b * b;
         }
         out[m] = sqrt(num) / sqrt(den);
+    }
+}
+
+/*
+ * Per-worker, per-tensor L2 norms (the parameter, update and gradient norms the paper plots
+ * for its billion-scale runs: additional-results appendix, figure on update and parameter
+ * norms; Section 6, RQ3, gradient norms after doubling the workers).  a is [M][stride] in
+ * fp64; tensor k of worker m occupies a[m*stride + offs[k] .. + numel[k]).  Writes
+ * out[m*num_tensors + k] = sqrt(sum of squares) and, if total_out is not NULL,
+ * total_out[m] = the norm over all tensors of worker m (elements between tensors are not read).
+ */
+void desloc_oracle_tensor_norms(int32_t M, int64_t stride, int32_t num_tensors, const int64_t *offs,
+                                const int64_t *numel, const double *a, double *out,
+                                double *total_out) {
+    for (int m = 0; m < M; ++m) {
+        double all = 0.0;
+        for (int32_t k = 0; k < num_tensors; ++k) {
+            double acc = 0.0;
+            for (int64_t i = 0; i < numel[k]; ++i) {
+                const double e = a[(int64_t)m * stride + offs[k] + i];
+                acc += e * e;
+            }
+            out[(int64_t)m * num_tensors + k] = sqrt(acc);
+            all += acc;
+        }
+        if (total_out) total_out[m] = sqrt(all);
     }
 }
 

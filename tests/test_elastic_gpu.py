@@ -61,11 +61,15 @@ def test_double_then_shrink_worker_count(name):
     ov = grow(ov) if ov is not None else None
     valid = st.valid_mask()
     after = [_host(b) for b in (st.x, st.u) + ((st.v,) if st.v is not None else ())]
-    for b4, aft in zip(before, after):
-        want = oracle.worker_mean(b4)
+    for b4, aft, ref in zip(before, after, (ox, ou) + ((ov,) if ov is not None else ())):
         assert np.array_equal(aft[:2], b4)                       # survivors untouched
-        for j in (2, 3):                                         # joiners = mean, bit for bit
+        # joiners hold the mean of the device's own survivors, rounded once (checked against the
+        # definition written out here: the oracle is never fed a value the device produced) ...
+        want = ((b4[0].astype(np.float64) + b4[1].astype(np.float64)) / 2.0).astype(np.float32)
+        for j in (2, 3):
             assert np.array_equal(aft[j][valid], want[valid])
+        # ... and agree with the oracle's own joiners, grown from the oracle's own trajectory
+        compare_per_tensor(st, aft, ref, "joiners")
     for t in range(6, 12):
         step(t)
     # ---- shrink: workers 1 and 3 leave; survivors keep their buffers

@@ -48,10 +48,8 @@ def test_normclip_step_matches_oracle(name, M, align):
         if mx >= 10.0:
             assert all(s == 1.0 for s in got_s[1:])       # worker 0 is blown up at t = 5
             assert (got_s[0] == 1.0) == (t != 5)
-        # the oracle steps with the fp32 factors the device used, so the comparison isolates
-        # the update; the factors themselves were checked just above
-        mo = oracle.step(ocfg, t, lr, ox, ou, ov, g_host, clip_bound=cb,
-                         gscale=np.asarray(got_s, dtype=np.float64))
+        # the oracle steps with its OWN fp64 factors: nothing read back from the device enters it
+        mo = oracle.step(ocfg, t, lr, ox, ou, ov, g_host, clip_bound=cb, gscale=scales)
         assert mk == mo
     torch.cuda.synchronize()
     compare_per_tensor(st, st.to_numpy(st.x), ox, "x")
@@ -83,16 +81,15 @@ def test_normclip_with_fp32_gradients(M):
             eng.step_normclip(t, f32r(w.lr), st.views(st.g), mx)
             got_n, got_s = eng.grad_norms()
             assert np.allclose(got_n, norms, rtol=2e-6) and np.allclose(got_s, scales, rtol=2e-6)
-            oracle.step(oracle_cfg(w), t, f32r(w.lr), ox, ou, ov, g_host,
-                        gscale=np.asarray(got_s, dtype=np.float64))
+            oracle.step(oracle_cfg(w), t, f32r(w.lr), ox, ou, ov, g_host, gscale=scales)
         torch.cuda.synchronize()
         compare_per_tensor(st, st.to_numpy(st.x), ox, "x")
         compare_per_tensor(st, st.to_numpy(st.v), ov, "v")
         eng.close()
 
 
-def test_normclip_end_to_end_against_oracle_factors():
-    """Same run but the oracle uses its own fp64 factors: the end state still meets the bar."""
+def test_normclip_workload4_recipe_with_decay():
+    """Workload 4's recipe (weight decay 0.1) with a bound that clips every step."""
     import paper_2505_22549_b200 as d
     w = di.mini(di.WORKLOADS["cfg4_adam_1p7b"], T=10).replace(K=(2, 3, 4))
     dev = torch.device("cuda:0")
@@ -137,7 +134,10 @@ def test_normclip_is_deterministic_and_rejects_bad_bounds():
 
 @pytest.mark.parametrize("opt", ["adam", "sgdm"])
 def test_rel_change_matches_oracle(opt):
-    """||s_{t+K} - s_t|| / ||s_t|| over K = 5 steps for x, u (and v)."""
+    """||s_{t+K} - s_t|| / ||s_t|| over K = 5 steps for x, u (and v).  The oracle measures its own
+    trajectory (same seeded inputs), never the device's buffers.  Both trajectories agree to
+    1e-5 of each tensor's scale, which bounds the difference of the two ratios r by
+    1e-5 (||now|| + ||then||) / ||then|| + 1e-5 r <= 2e-5 (1 + r); the assertion allows 3e-5 (1 + r)."""
     import paper_2505_22549_b200 as d
     w = di.mini(di.WORKLOADS[f"cfg5_{opt}_desloc"], T=8).replace(M=3, K=(2, 3, 4))
     dev = torch.device("cuda:0")
@@ -145,21 +145,25 @@ def test_rel_change_matches_oracle(opt):
         st = State(w, dev, align=align)
         eng = make_engine(d, w, st)
         valid = _valid(st)
-        snaps = None
+        ox, ou = st.to_numpy(st.x), st.to_numpy(st.u)          # initial state, before any step
+        ov = st.to_numpy(st.v) if st.v is not None else None
+        ocfg = oracle_cfg(w)
+        snaps = osnaps = None
         for t in range(w.T):
             if t == 3:
                 snaps = [[b.clone() for b in bufs] if bufs is not None else None
                          for bufs in (st.x, st.u, st.v)]
+                osnaps = [a.copy() if a is not None else None for a in (ox, ou, ov)]
             st.fill_grads(t)
             eng.step(t, f32r(w.lr), st.views(st.g))
+            oracle.step(ocfg, t, f32r(w.lr), ox, ou, ov, st.to_numpy(st.g))
         torch.cuda.synchronize()
-        arrays = [(0, st.x), (1, st.u)] + ([(2, st.v)] if st.v is not None else [])
-        for idx, bufs in arrays:
-            got = eng.rel_change(idx, st.views(snaps[idx]))
-            now = np.ascontiguousarray(st.to_numpy(bufs)[:, valid])
-            then = np.ascontiguousarray(st.to_numpy(snaps[idx])[:, valid])
-            want = oracle.rel_change(now, then)
-            assert np.allclose(got, want, rtol=5e-6), (idx, got, want)
+        arrays = [(0, ox), (1, ou)] + ([(2, ov)] if ov is not None else [])
+        for idx, onow in arrays:
+            got = np.asarray(eng.rel_change(idx, st.views(snaps[idx])), dtype=np.float64)
+            want = oracle.rel_change(np.ascontiguousarray(onow[:, valid]),
+                                     np.ascontiguousarray(osnaps[idx][:, valid]))
+            assert np.all(np.abs(got - want) <= 3e-5 * (1.0 + want)), (idx, got, want)
             assert min(want) > 0
         if st.v is None:
             with pytest.raises(d.DeslocError):

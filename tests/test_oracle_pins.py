@@ -596,3 +596,106 @@ def test_adopt_normalised_gradient_clip_is_two_sided():
     x, u, v = zeros(1, 3), zeros(1, 3), zeros(1, 3)
     oracle.step(cfg, 0, 1.0, x, u, v, f32([[4.0, -4.0, 0.5]]), clip_bound=0.0)
     assert np.array_equal(u[0], f32([0.0, 0.0, 0.0])) and np.all(v[0] > 0)
+
+
+# --------------------------------------------------------------------------- update d_t and norms
+def test_update_d_matches_hand_examples():
+    """d_t from the oracle against the hand examples, two ways: as eta u_t / sqrt(v_t) (eta u_t
+    for ADOPT and SGDM) evaluated from the golden states, and as the difference between the base
+    the step starts from (the worker's own x_t, or the mean on an x-sync step) and the golden
+    x_{t+1}."""
+    gold = json.load(open(GOLD))
+    cases = [
+        ("adam", ADAM, dict(beta1=0.5, beta2=0.5, eps=0.0), "u", 0.0),
+        ("adopt", ADOPT, dict(beta1=0.5, beta2=0.5, eps=1e-6), "m", 1.0),
+        ("sgdm", SGDM, dict(beta1=0.5), "u", None),
+    ]
+    for key, opt, hp, uname, v_init in cases:
+        ex = gold[key]
+        Kv = ex.get("Kv", 0)
+        cfg = oracle.make_cfg(2, opt, Kx=ex["Kx"], Ku=ex.get("Ku", ex.get("Km")), Kv=Kv, **hp)
+        x, u = f32([[1.0], [1.0]]), zeros(2, 1)
+        v = None if v_init is None else f32([[v_init], [v_init]])
+        num = lambda s: float(Fraction(s)) if isinstance(s, str) else float(s)
+        prev_x = [1.0, 1.0]
+        for t, g in enumerate(ex["g"]):
+            d = np.zeros((2, 1), dtype=np.float64)
+            mask = oracle.step(cfg, t, 0.1, x, u, v, f32([[num(g[0])], [num(g[1])]]), d_out=d)
+            base = [sum(prev_x) / 2.0] * 2 if mask & SYNC_X else prev_x
+            for m in range(2):
+                un = num(ex[uname][t][m])
+                want = 0.1 * un / math.sqrt(num(ex["v"][t][m])) if opt == ADAM else 0.1 * un
+                assert abs(d[m, 0] - want) < 2e-7, (key, t, m)
+                assert abs(d[m, 0] - (base[m] - num(ex["x"][t][m]))) < 5e-7, (key, t, m)
+            prev_x = [num(ex["x"][t][m]) for m in range(2)]
+
+
+def test_update_d_is_the_parameter_change_of_torch_adamw_without_the_decay_term():
+    """M = 1 against torch.optim.AdamW in fp64: with decay factor (1 - eta wd) applied to the
+    parameter first, what remains of the library's parameter change is d_t."""
+    rng = np.random.default_rng(5)
+    n, T, lr, b1, b2, wd = 40, 12, 1e-2, 0.9, 0.99, 0.1
+    x0 = rng.normal(size=n).astype(np.float32)
+    grads = rng.normal(size=(T, n)).astype(np.float32)
+    p = torch.nn.Parameter(torch.tensor(x0, dtype=torch.float64))
+    opt = torch.optim.AdamW([p], lr=lr, betas=(b1, b2), eps=0.0, weight_decay=wd)
+    cfg = oracle.make_cfg(1, ADAM, beta1=b1, beta2=b2, eps=0.0, weight_decay=wd, Kx=2, Ku=3, Kv=4)
+    x, u, v = f32(x0[None]), zeros(1, n), zeros(1, n)
+    for t in range(T):
+        eta_t = lr * math.sqrt(1 - b2 ** (t + 1)) / (1 - b1 ** (t + 1))
+        opt.param_groups[0]["weight_decay"] = wd * eta_t / lr
+        p.grad = torch.tensor(grads[t], dtype=torch.float64)
+        before = p.detach().clone()
+        opt.step()
+        d_lib = (before * (1.0 - eta_t * wd) - p.detach()).numpy()
+        d = np.zeros((1, n), dtype=np.float64)
+        oracle.step(cfg, t, eta_t, x, u, v, f32(grads[t][None]), d_out=d)
+        # the oracle's u, v are re-read from fp32 storage every step: agreement to ~1e-6 relative
+        assert np.max(np.abs(d[0] - d_lib)) < 2e-6 * np.max(np.abs(d_lib))
+        assert np.max(np.abs(d_lib)) > 1e-3
+
+
+def test_update_d_one_step_closed_forms():
+    """From zero states one step gives u = (1-b1) g, v = (1-b2) g^2, so
+    Adam d = eta (1-b1) g / sqrt((1-b2) g^2 + lambda^2), SGDM d = eta (1-b) g, and ADOPT (seeded
+    v = 4, so the normaliser is 2) d = eta (1-b1) g / 2; weight decay does not enter d."""
+    g = np.array([[3.0, -0.5, 0.25]], dtype=np.float32)
+    g64 = g.astype(np.float64)
+    for opt, want in (
+        (ADAM, 0.1 * 0.25 * g64 / np.sqrt(0.5 * g64 ** 2 + 0.125 ** 2)),
+        (SGDM, 0.1 * 0.25 * g64),
+        (ADOPT, 0.1 * 0.25 * g64 / 2.0),
+    ):
+        cfg = oracle.make_cfg(1, opt, beta1=0.75, beta2=0.5, eps=0.125 if opt == ADAM else 1e-6,
+                              weight_decay=0.3)
+        x, u = f32([[1.0, 2.0, 3.0]]), zeros(1, 3)
+        v = None if opt == SGDM else (f32([[4.0, 4.0, 4.0]]) if opt == ADOPT else zeros(1, 3))
+        d = np.full((1, 3), np.nan)
+        oracle.step(cfg, 0, 0.1, x, u, v, g.copy(), d_out=d)
+        assert np.allclose(d, want, rtol=1e-13, atol=0)
+        # and x moved by the decay plus d
+        assert np.allclose(x, np.array([[1.0, 2.0, 3.0]]) * (1 - 0.1 * 0.3) - want, rtol=2e-7)
+
+
+def test_tensor_norms_closed_forms_and_library():
+    """3-4-5 and 5-12-13 triples in separate tensors with padding between them (padding holds
+    garbage that must not be read), whole-model norm = sqrt of the sum of squares, and a random
+    case against numpy.linalg.norm."""
+    a = np.full((2, 12), 1e6, dtype=np.float32)
+    offs, numel = [1, 4, 8], [2, 3, 1]
+    a[0, 1:3] = [3, 4];  a[0, 4:7] = [0, -5, 12];  a[0, 8] = -2
+    a[1, 1:3] = [0, 0];  a[1, 4:7] = [1, 2, 2];    a[1, 8] = 7
+    per, tot = oracle.tensor_norms(a, offs, numel)
+    assert np.array_equal(per, [[5.0, 13.0, 2.0], [0.0, 3.0, 7.0]])
+    assert np.allclose(tot, [math.sqrt(25 + 169 + 4), math.sqrt(9 + 49)], rtol=1e-15)
+    rng = np.random.default_rng(9)
+    b = rng.normal(size=(3, 1000))
+    offs, numel = [0, 10, 500, 999], [10, 400, 499, 1]
+    per, tot = oracle.tensor_norms(b, offs, numel)
+    for m in range(3):
+        for k, (o, c) in enumerate(zip(offs, numel)):
+            assert abs(per[m, k] - np.linalg.norm(b[m, o:o + c])) < 1e-12 * (1 + per[m, k])
+        want = np.linalg.norm(np.concatenate([b[m, o:o + c] for o, c in zip(offs, numel)]))
+        assert abs(tot[m] - want) < 1e-12 * want
+    with pytest.raises(ValueError):
+        oracle.tensor_norms(b, [990], [11])
