@@ -3,6 +3,11 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
 
+With --gpus N > 1 and no torchrun environment the program starts N ranks of itself (one per
+GPU); under torchrun it is one of the ranks.  After the headline workload (default: workload 4)
+the single-GPU run times every other workload of the benchmark definition and reports them in
+"all_configs".
+
 One "step" is one call of desloc_step(): the whole hot path (clip, desynced averaging,
 optimizer update for all M worker replicas) over the full synthetic parameter/gradient set.
 Steps run t = 0, 1, 2, ... under the workload's own (K_x, K_u, K_v), so the timed region mixes
@@ -200,10 +205,221 @@ def run_reference(args, w):
 
 
 # ------------------------------------------------------------------------------ GPU leg
+class Resident:
+    """One workload resident in HBM: M replicas of x, u, v, one gradient set, and views per
+    tensor.  torch is used for the memory and the stream only."""
+
+    def __init__(self, w, dev, rank=0):
+        import torch
+        import desloc_inputs as di
+        self.w, self.dev = w, dev
+        align = 4
+        self.nflat = di.flat_size(w.numel, align)
+        self.offs = di.offsets_of(w.numel, align)
+        gdt = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
+        x0 = di.init_params(w.replace(seed=w.seed + rank), device=dev, align=align)
+        self.X = [x0.clone() for _ in range(w.M - 1)] + [x0]
+        self.U = [torch.zeros(self.nflat, dtype=torch.float32, device=dev) for _ in range(w.M)]
+        self.V = [torch.zeros(self.nflat, dtype=torch.float32, device=dev) for _ in range(w.M)] \
+            if w.opt != "sgdm" else None
+        self.G = [torch.empty(self.nflat, dtype=gdt, device=dev) for _ in range(w.M)]
+        for m in range(w.M):
+            di.fill_grads_(w.replace(seed=w.seed + rank), 0, m, self.G[m], align=align)
+
+    def views(self, bufs):
+        return [[b[o:o + n] for o, n in zip(self.offs, self.w.numel)] for b in bufs]
+
+    def engine(self, d, w=None, post=False):
+        w = w or self.w
+        flags = d.DESLOC_FLAG_ADOPT_NORM_CLIP if w.adopt_norm_clip else 0
+        if post:
+            flags |= d.DESLOC_FLAG_POST_AVERAGE
+        return d.DesLoc(self.views(self.X), self.views(self.U),
+                        self.views(self.V) if self.V is not None else None, opt=w.opt,
+                        grad_dtype=w.grad_dtype, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
+                        weight_decay=w.weight_decay, clip_rho=w.clip_rho, K=w.K, flags=flags)
+
+
+def timed_loop(stream, fn, reps):
+    """CUDA-event time per call of fn over `reps` back-to-back calls, in ms."""
+    import torch
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(reps):
+        fn()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def rates(w, ms, peak, nbytes=None):
+    nbytes = nbytes if nbytes is not None else w.M * w.N * bytes_per_param(w)
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"ms": ms, "gups": w.M * w.N / (ms * 1e-3) / 1e9, "gbs": gbs,
+            "frac_of_measured_peak": gbs / peak, "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS}
+
+
+def per_mask_and_variants(w, eng, g, stream, peak, reps):
+    """Local, x-only and all-sync steps timed in isolation, then the norm-clipped step (one more
+    read of the gradients) and the diagnostics step (same bytes as the plain step)."""
+    out = {"by_mask": {}}
+    for mk in [0, 1, 3 if w.opt == "sgdm" else 7]:
+        if w.M == 1 and mk:
+            continue
+        fn = lambda: eng.step_masked(mk, w.lr, g, clip_bound=1.0)
+        fn(); fn()
+        out["by_mask"][str(mk)] = rates(w, timed_loop(stream, fn, reps), peak)
+    gbytes = 2 if w.grad_dtype == "bf16" else 4
+    fn = lambda: eng.step_normclip(1, w.lr, g, 1.0, clip_bound=1.0)
+    fn(); fn()
+    nc_bytes = w.M * w.N * (bytes_per_param(w) + gbytes)
+    out["normclip_step"] = dict(rates(w, timed_loop(stream, fn, reps), peak, nc_bytes),
+                                launches_per_step=3, algorithmic_bytes=nc_bytes)
+    fn = lambda: eng.step_diag(1, w.lr, g, clip_bound=1.0)
+    fn(); fn()
+    out["diag_step"] = dict(rates(w, timed_loop(stream, fn, reps), peak),
+                            note="same step, plus per-(worker, tensor) norms of g, x, d fused in")
+    return out
+
+
+def graph_window(w, eng, g, stream, eager_us):
+    """Small, launch-bound workloads: a CUDA graph of one lcm(K) window of steps."""
+    import math
+    import torch
+    L = math.lcm(*[k for k in w.K if k > 0])
+    if L > 256:
+        return None
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(stream)
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for t in range(L):
+                eng.step(t, w.lr, g, clip_bound=w.clip_bound(t))
+    stream.wait_stream(side)
+    for _ in range(3):
+        graph.replay()
+    us = timed_loop(stream, graph.replay, 50) * 1e3 / L
+    return {"window_steps": L, "us_per_step": us, "gups": w.M * w.N / (us * 1e-6) / 1e9,
+            "eager_us_per_step": eager_us}
+
+
+PARITY_TESTS = {
+    "cfg1_adam_n4096": "tests/test_parity_gpu.py::test_cfg1_adam_n4096_full_run (every element, T = 64)",
+    "cfg2_adam_135m": "tests/test_parity_fullsize_gpu.py::test_fullsize_sampled_parity[cfg2_adam_135m-*]",
+    "cfg3_adopt_360m": "tests/test_parity_fullsize_gpu.py::test_fullsize_sampled_parity[cfg3_adopt_360m-*]",
+    "cfg4_adam_1p7b": "tests/test_parity_fullsize_gpu.py::test_fullsize_sampled_parity[cfg4_adam_1p7b-*]",
+}
+
+
+def parity_test_of(name):
+    """The -m gpu test that checks this workload at full size, in this launch configuration,
+    against the oracle (this program may run the oracle only for its CPU-baseline leg)."""
+    return PARITY_TESTS.get(
+        name, f"tests/test_parity_fullsize_gpu.py::test_fullsize_sampled_parity[{name}-*]")
+
+
+def time_config(d, w, res, steps, warmup, peak, rank=0, world=1, barrier=None, sampler=None,
+                post=False):
+    """The timed region of one workload: exactly `steps` steps under its own schedule, placed so
+    that an x-sync step falls inside; then the per-mask and variant timings."""
+    import torch
+    dev = res.dev
+    stream = torch.cuda.current_stream(dev)
+    eng = res.engine(d, w, post)
+    g = eng.bind_grads(res.views(res.G))
+    step = lambda t: eng.step(t, w.lr, g, clip_bound=w.clip_bound(t))
+    t_next = 0
+    for _ in range(max(3, warmup)):
+        step(t_next); t_next += 1
+    barrier()
+    Kx = w.K[0]
+    if Kx > 1:
+        t_next = max(t_next, (t_next // Kx + 1) * Kx - steps // 2)
+    if sampler is not None:
+        sampler.start()
+        time.sleep(0.3)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    masks = []
+    launches0 = eng.launches()
+    barrier()
+    wall0 = time.time()
+    ev[0].record(stream)
+    for i in range(steps):
+        masks.append(step(t_next)); t_next += 1
+        ev[i + 1].record(stream)
+    barrier()
+    wall1 = time.time()
+    launches = eng.launches() - launches0
+    total_ms = ev[0].elapsed_time(ev[-1])
+    per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+    clocks = sampler.stop(wall0, wall1) if sampler is not None else None
+    total_ms = d.dist.max_over_ranks(total_ms, dev)
+    launches = d.dist.sum_over_ranks(launches, dev)
+    out = {"eng": eng, "g": g, "masks": masks, "per_step": per_step, "total_ms": total_ms,
+           "launches": launches, "clocks": clocks,
+           "value": world * w.M * w.N * steps / (total_ms * 1e-3) / 1e9}
+    out.update(per_mask_and_variants(w, eng, g, stream, peak, max(3, min(steps, 10))))
+    return out
+
+
+def config_entry(w, r, steps):
+    ms = r["total_ms"] / steps
+    e = {"workload": w.name, "opt": w.opt, "M": w.M, "params": w.N, "K": list(w.K),
+         "grad_dtype": w.grad_dtype, "steps": steps, "ms_per_step": ms, "value": r["value"],
+         "unit": UNIT, "masks_in_timed_region": r["masks"], "by_mask": r["by_mask"],
+         "normclip_step": r["normclip_step"], "diag_step": r["diag_step"],
+         "parity_test": parity_test_of(w.name)}
+    gbs = w.M * w.N * bytes_per_param(w) / (ms * 1e-3) / 1e9
+    e["gbs"] = gbs
+    e["frac_of_nominal_8tbs"] = gbs / NOMINAL_HBM_GBS
+    return e
+
+
+def run_all_configs(d, dev, steps, warmup, peak, skip):
+    """Every other workload of the benchmark definition, one after the other on the same GPU:
+    workload 1 (latency-bound: eager and CUDA-graph microseconds per step), workload 2,
+    workload 3, and workload 5's two optimizers under its three schedules."""
+    import torch
+    import desloc_inputs as di
+    stream = torch.cuda.current_stream(dev)
+    out = []
+    no_barrier = torch.cuda.synchronize
+    groups = [["cfg1_adam_n4096"], ["cfg2_adam_135m"], ["cfg3_adopt_360m"], ["cfg4_adam_1p7b"],
+              ["cfg5_sgdm_ddp", "cfg5_sgdm_local", "cfg5_sgdm_desloc"],
+              ["cfg5_adam_ddp", "cfg5_adam_local", "cfg5_adam_desloc"]]
+    for names in groups:
+        names = [n for n in names if n != skip]
+        if not names:
+            continue
+        w0 = di.WORKLOADS[names[0]]
+        free, _ = torch.cuda.mem_get_info(dev)
+        need = w0.N * w0.M * (14 if w0.opt != "sgdm" else 10) + (4 << 30)
+        if free < need:
+            out += [{"workload": n, "skipped": f"needs {need >> 30} GiB, {free >> 30} GiB free"}
+                    for n in names]
+            continue
+        res = Resident(w0, dev)            # the schedules of a group share one resident state
+        for n in names:
+            w = di.WORKLOADS[n]
+            r = time_config(d, w, res, steps, warmup, peak, barrier=no_barrier)
+            e = config_entry(w, r, steps)
+            e["frac_of_measured_peak"] = e["gbs"] / peak
+            if w.M * w.N * 14 < (126 << 20) and w.M * len(w.numel) <= 32 and min(w.K) > 0:
+                e["graph_window"] = graph_window(w, r["eng"], r["g"], stream,
+                                                 r["total_ms"] * 1e3 / steps)
+                e["note"] = "fits in L2: latency-bound, microseconds per step are the figure"
+            r["eng"].close()
+            out.append(e)
+        del res, r
+        torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args, w):
     import torch
     import torch.distributed as dist
-    import desloc_inputs as di
     import paper_2505_22549_b200 as d
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -221,145 +437,23 @@ def run_ours(args, w):
             dist.barrier()
         torch.cuda.synchronize()
 
+    peak, peak_kind = measured_peak()
     # ---- resident state: every rank holds its own M replicas of the whole tensor list -------
-    align = 4
-    nflat = di.flat_size(w.numel, align)
-    offs = di.offsets_of(w.numel, align)
-    gdt = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
-    x0 = di.init_params(w.replace(seed=w.seed + rank), device=dev, align=align)
-    X = [x0.clone() for _ in range(w.M - 1)] + [x0]
-    U = [torch.zeros(nflat, dtype=torch.float32, device=dev) for _ in range(w.M)]
-    V = [torch.zeros(nflat, dtype=torch.float32, device=dev) for _ in range(w.M)] \
-        if w.opt != "sgdm" else None
-    G = [torch.empty(nflat, dtype=gdt, device=dev) for _ in range(w.M)]
-    for m in range(w.M):
-        di.fill_grads_(w.replace(seed=w.seed + rank), 0, m, G[m], align=align)
-    views = lambda bufs: [[b[o:o + n] for o, n in zip(offs, w.numel)] for b in bufs]
-    flags = d.DESLOC_FLAG_ADOPT_NORM_CLIP if w.adopt_norm_clip else 0
-    if args.post_average:
-        flags |= d.DESLOC_FLAG_POST_AVERAGE
-    eng = d.DesLoc(views(X), views(U), views(V) if V is not None else None, opt=w.opt,
-                   grad_dtype=w.grad_dtype, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
-                   weight_decay=w.weight_decay, clip_rho=w.clip_rho, K=w.K, flags=flags)
-    if args.ctas_per_sm is not None:
-        eng.set_launch_shape(args.ctas_per_sm)
-    gv = views(G)
+    res = Resident(w, dev, rank)
     bpp = bytes_per_param(w)
     launch_bytes = w.M * w.N * bpp
     stream = torch.cuda.current_stream(dev)
+    r = time_config(d, w, res, args.steps, args.warmup, peak, rank, world, barrier,
+                    ClockSampler(local_rank) if rank == 0 else None, args.post_average)
+    eng, g = r["eng"], r["g"]
 
-    def step(t):
-        return eng.step(t, w.lr, gv, clip_bound=w.clip_bound(t))
-
-    # ---- warm-up: t = 0 (all arrays sync) onwards ---------------------------------------------
-    t_next = 0
-    for _ in range(max(3, args.warmup)):
-        step(t_next); t_next += 1
-    barrier()
-    # the timed window is placed so that one x-sync step falls in its middle, as in a real run
-    Kx = w.K[0]
-    if Kx > 1:
-        t_next = max(t_next, (t_next // Kx + 1) * Kx - args.steps // 2)
-
-    # ---- timed region: exactly K steps, CUDA events on the launching stream -------------------
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.3)
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-    masks = []
-    launches0 = eng.launches()
-    barrier()
-    wall0 = time.time()
-    ev[0].record(stream)
-    for i in range(args.steps):
-        masks.append(step(t_next)); t_next += 1
-        ev[i + 1].record(stream)
-    barrier()
-    wall1 = time.time()
-    launches = eng.launches() - launches0
-    total_ms = ev[0].elapsed_time(ev[-1])
-    per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
-    clocks = sampler.stop(wall0, wall1) if rank == 0 else None
-    # every multi-GPU number is the slowest rank's; launches add up (helpers covered by the
-    # world-size-2 gloo tests)
-    total_ms = d.dist.max_over_ranks(total_ms, dev)
-    launches = d.dist.sum_over_ranks(launches, dev)
-    value = world * w.M * w.N * args.steps / (total_ms * 1e-3) / 1e9
-
-    # ---- per-mask timing (outside the headline region): local, x-only, all-sync ---------------
-    by_mask = {}
-    peak, peak_kind = measured_peak()
-    masks_to_time = [0, 1, 3 if w.opt == "sgdm" else 7]
-    reps = max(3, min(args.steps, 10))
-    for mk in masks_to_time:
-        if w.M == 1 and mk:
-            continue
-        for _ in range(2):
-            eng.step_masked(mk, w.lr, gv, clip_bound=1.0)
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(reps):
-            eng.step_masked(mk, w.lr, gv, clip_bound=1.0)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1) / reps
-        gbs = launch_bytes / (ms * 1e-3) / 1e9
-        by_mask[str(mk)] = {"ms": ms, "gups": w.M * w.N / (ms * 1e-3) / 1e9, "gbs": gbs,
-                            "frac_of_measured_peak": gbs / peak,
-                            "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS}
-
-    # ---- norm-based clipping in front of the step (reads the gradients once more) ------------
-    gbytes = 2 if w.grad_dtype == "bf16" else 4
-    for _ in range(2):
-        eng.step_normclip(1, w.lr, gv, 1.0, clip_bound=1.0)
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(reps):
-        eng.step_normclip(1, w.lr, gv, 1.0, clip_bound=1.0)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / reps
-    nc_bytes = w.M * w.N * (bpp + gbytes)
-    normclip = {"ms": ms, "gups": w.M * w.N / (ms * 1e-3) / 1e9,
-                "gbs": nc_bytes / (ms * 1e-3) / 1e9,
-                "frac_of_measured_peak": nc_bytes / (ms * 1e-3) / 1e9 / peak,
-                "launches_per_step": 3, "algorithmic_bytes": nc_bytes}
-
-    # ---- small, launch-bound workloads: a CUDA graph of one lcm(K) window of steps -----------
-    graph_info = None
     resident = w.M * w.N * (bpp - (8 if w.opt == "sgdm" else 12))
+    graph_info = None
     if resident < (126 << 20) and w.M * len(w.numel) <= 32 and min(w.K) > 0:
-        import math
-        L = math.lcm(*[k for k in w.K if k > 0])
-        if L <= 256:
-            graph = torch.cuda.CUDAGraph()
-            side = torch.cuda.Stream()
-            side.wait_stream(stream)
-            with torch.cuda.stream(side):
-                with torch.cuda.graph(graph, stream=side):
-                    for t in range(L):
-                        eng.step(t, w.lr, gv, clip_bound=w.clip_bound(t))
-            stream.wait_stream(side)
-            for _ in range(3):
-                graph.replay()
-            torch.cuda.synchronize()
-            nrep = 50
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-            for _ in range(nrep):
-                graph.replay()
-            e1.record(stream)
-            torch.cuda.synchronize()
-            us = e0.elapsed_time(e1) * 1e3 / (nrep * L)
-            graph_info = {"window_steps": L, "us_per_step": us,
-                          "gups": w.M * w.N / (us * 1e-6) / 1e9,
-                          "eager_us_per_step": total_ms * 1e3 / args.steps}
+        graph_info = graph_window(w, eng, g, stream, r["total_ms"] * 1e3 / args.steps)
 
     # ---- roofline of the dominant kernel (the local-step kernel), from the timed region -------
-    local_ms = [ms for ms, mk in zip(per_step, masks) if mk == 0] or per_step
+    local_ms = [ms for ms, mk in zip(r["per_step"], r["masks"]) if mk == 0] or r["per_step"]
     avg_local_ms = float(np.mean(local_ms))
     achieved = launch_bytes / (avg_local_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
@@ -374,7 +468,17 @@ def run_ours(args, w):
                 "avg_launch_ms": avg_local_ms, "launches_averaged": len(local_ms)}
 
     # ---- end to end: gradients start in pinned host memory, a result is read back -------------
-    e2e = None if args.skip_e2e else run_e2e(args, w, eng, G, X, offs, dev, world, barrier)
+    e2e = None if args.skip_e2e else run_e2e(args, w, eng, res.G, res.X, res.offs, dev, world, barrier)
+    eng.close()
+    headline = config_entry(w, r, args.steps)
+    value, total_ms, launches, clocks = r["value"], r["total_ms"], r["launches"], r["clocks"]
+    del res, r, eng, g
+    torch.cuda.empty_cache()
+
+    all_configs = None
+    if rank == 0 and world == 1 and not args.skip_all_configs:
+        all_configs = run_all_configs(d, dev, max(4, min(args.steps, 20)), args.warmup, peak,
+                                      skip=w.name)
 
     if rank == 0:
         cpu = (time_oracle(w, seconds_target=15.0) if not args.skip_cpu else
@@ -388,19 +492,21 @@ def run_ours(args, w):
             "data": "synthetic",
             "config": {"workload": w.name, "opt": w.opt, "M": w.M, "params": w.N,
                        "tensors": len(w.numel), "grad_dtype": w.grad_dtype, "K": list(w.K),
-                       "resident_gb": w.M * w.N * (bpp - (8 if w.opt == "sgdm" else 12)) / 1e9,
+                       "resident_gb": resident / 1e9,
                        "l2": ("inputs larger than L2 (no flush needed)" if resident > (126 << 20)
                               else "workload fits in L2: latency-bound, see graph_window"),
                        "parallelism": f"{world} independent replica set(s), no collective",
                        "ordering": "post-average" if args.post_average else "pre-average",
-                       "masks_in_timed_region": masks},
-            "roofline": roofline, "by_mask": by_mask, "normclip_step": normclip, "graph_window": graph_info, "cpu_baseline": {k: cpu[k] for k in
-                                                                       ("value", "unit", "cores", "kind", "sample",
-                                                                        "single_thread") if k in cpu},
-            "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+                       "masks_in_timed_region": headline["masks_in_timed_region"],
+                       "parity_test": headline["parity_test"]},
+            "roofline": roofline, "by_mask": headline["by_mask"],
+            "normclip_step": headline["normclip_step"], "diag_step": headline["diag_step"],
+            "graph_window": graph_info,
+            "cpu_baseline": {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample",
+                                                 "single_thread") if k in cpu},
+            "e2e": e2e, "gpu_launches": launches, "clocks": clocks, "all_configs": all_configs,
         }
         print(json.dumps(line), flush=True)
-    eng.close()
     if world > 1:
         dist.destroy_process_group()
     return 0
@@ -472,34 +578,40 @@ def run_e2e(args, w, eng, G, X, offs, dev, world, barrier):
                     + ("" if share else " (one host buffer re-sent for each worker)")}
 
 
-def main():
+def launcher_command(gpus: int, argv, port: int | None = None):
+    """The command that starts `gpus` ranks of this program on this node (one process per GPU,
+    rendezvous on 127.0.0.1), as the benchmark contract launches it."""
+    if port is None:
+        import socket
+        with socket.socket() as s:
+            s.bind(("127.0.0.1", 0))
+            port = s.getsockname()[1]
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port),
+            os.path.abspath(__file__)] + list(argv)
+
+
+def main(argv=None):
+    argv = sys.argv[1:] if argv is None else list(argv)
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4_adam_1p7b")
-    ap.add_argument("--ctas-per-sm", type=int, default=None)
-    ap.add_argument("--workers", type=int, default=None,
-                    help="override the workload's worker count M (exploration only)")
     ap.add_argument("--post-average", action="store_true",
                     help="average after the update (ordering of Algorithms 4-5) instead of before")
-    ap.add_argument("--grad-dtype", default=None, choices=["f32", "bf16"],
-                    help="override the workload's gradient dtype (exploration only)")
-    ap.add_argument("--opt", default=None, choices=["adam", "adopt", "sgdm"],
-                    help="override the workload's optimizer (exploration only)")
     ap.add_argument("--skip-e2e", action="store_true", help="omit the host-buffer leg (profiling)")
     ap.add_argument("--skip-cpu", action="store_true", help="omit the CPU oracle leg (profiling)")
-    args = ap.parse_args()
+    ap.add_argument("--skip-all-configs", action="store_true",
+                    help="time the named workload only, not the other workloads after it")
+    args = ap.parse_args(argv)
     import desloc_inputs as di
     w = di.WORKLOADS[args.workload]
-    if args.workers:
-        w = w.replace(name=f"{w.name}_M{args.workers}", M=args.workers)
-    if args.grad_dtype:
-        w = w.replace(name=f"{w.name}_{args.grad_dtype}", grad_dtype=args.grad_dtype)
-    if args.opt:
-        w = w.replace(name=f"{w.name}_{args.opt}", opt=args.opt,
-                      adopt_norm_clip=(args.opt == "adopt"))
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain program: become N ranks, one per GPU (replicas only, no collective
+        # on the data path; NCCL carries the barrier and the max over ranks of the timing)
+        return subprocess.call(launcher_command(args.gpus, argv))
     if args.impl == "reference":
         return run_reference(args, w)
     return run_ours(args, w)

@@ -169,8 +169,8 @@ DESLOC_API int desloc_step_masked(desloc_ctx *ctx, uint32_t mask, float lr_t, fl
 /*
  * One step with norm-based gradient clipping in front: worker m's whole gradient (all tensors)
  * is scaled by min(1, max_norm / ||g^m||_2) before the coordinate clip and the update.  This
- * is the clipping the paper's language-model runs used (model table in the experimental
- * details: "norm-based gradient clipping with clip-bound rho", rho = 1.0); Algorithms 1-3
+ * is how the paper's language-model runs clipped (the model table of the experimental-details
+ * appendix gives the bound on the gradient's L2 norm, 1.0, in its rho column); Algorithms 1-3
  * only have the coordinate-wise clip.  Costs one more read of the gradients: two reduction
  * launches (per-chunk partial sums in fp32, per-worker totals in fp64, fixed order, no
  * atomics) ahead of the step kernel, all enqueued on `stream` without host synchronisation.
@@ -186,6 +186,37 @@ DESLOC_API int desloc_step_normclip(desloc_ctx *ctx, int64_t t, float lr_t, floa
  * it: this call synchronises.
  */
 DESLOC_API int desloc_get_grad_norms(desloc_ctx *ctx, float *norms_out, float *scales_out,
+                                     void *stream);
+
+/*
+ * One step that also measures, per worker and per tensor, the L2 norms of
+ *   kind 0: the gradient g_t^m as read (before any clipping),
+ *   kind 1: the new parameters x_{t+1}^m as stored,
+ *   kind 2: the update d_t^m of Algorithms 2-3 (eta_t u_t / sqrt(v_t + lambda^2) for Adam,
+ *           eta_t u_t for ADOPT and SGDM; the weight-decay term is not part of it)
+ * -- the gradient, parameter and update norms the paper tracks (gradient norms after the
+ * workers are doubled, Section 6, RQ3; update and parameter norms of the billion-scale runs,
+ * additional-results appendix).  The step kernel already holds all three in registers, so the
+ * sums of squares are formed there, one partial per (kind, worker, chunk): no extra pass over
+ * memory, and the step computes exactly what desloc_step() computes.
+ *   max_norm : > 0 puts norm-based clipping in front as desloc_step_normclip() does; 0 = off.
+ * Other arguments as desloc_step().  Not available with desloc_step_host().
+ */
+DESLOC_API int desloc_step_diag(desloc_ctx *ctx, int64_t t, float lr_t, float clip_bound_t,
+                                float max_norm, const void *const *grads, void *stream,
+                                uint32_t *mask_out);
+
+/*
+ * Norms of the latest desloc_step_diag():
+ *   per_tensor_out : host, [3][M][num_tensors] floats, entry (kind * M + m) * num_tensors + k,
+ *                    or NULL;
+ *   total_out      : host, [3][M] floats, the norm over the whole tensor list, or NULL.
+ * Per-chunk partials are fp32; they are added per tensor, and the tensors per worker, in fp64
+ * in a fixed order (deterministic, no atomics).  Two small launches on `stream`, then the
+ * copies; the call waits for `stream`.  DESLOC_E_INVALID if no diagnostics step has run since
+ * the context was created or its workers were changed.
+ */
+DESLOC_API int desloc_get_diag_norms(desloc_ctx *ctx, float *per_tensor_out, float *total_out,
                                      void *stream);
 
 /*
@@ -224,15 +255,9 @@ DESLOC_API int desloc_destroy(desloc_ctx *ctx);
    distributed run of the same schedule would pay; Section 5.1 "Metrics"). */
 DESLOC_API int desloc_get_counters(const desloc_ctx *ctx, int64_t out[4]);
 
-/* Kernels launched by this context so far (one per step on the main path). */
+/* Kernels launched by this context so far (one per step on the main path, one thread block
+   per chunk). */
 DESLOC_API int64_t desloc_get_launch_count(const desloc_ctx *ctx);
-
-/*
- * Grid shape of the step kernel: ctas_per_sm = 0 (default) launches one thread block per work
- * item (a chunk, or a (worker, chunk) pair on local steps); 1..32 launches a persistent grid
- * of that many blocks per SM which stride over the items.  Results do not depend on it.
- */
-DESLOC_API int desloc_set_launch_shape(desloc_ctx *ctx, int32_t ctas_per_sm);
 
 /*
  * Multi-tensor plan: how the tensor list is cut into the fixed-size chunks that thread
@@ -259,26 +284,41 @@ DESLOC_API int64_t desloc_chunk_elems(void);
  * synchronisation that cudaMalloc and cudaFree bring.  This entry point needs no context and
  * calls no cudaMalloc, cudaFree, cudaMallocHost or any other allocating routine: its tables
  * go into a fixed array inside the library image, DESLOC_STATIC_SCRATCH_BYTES (about 320 KB)
- * of device memory that every GPU which loads the library holds until the process exits.
+ * of device memory per GPU, held until the process exits.
  *
  * Limits: M * num_tensors <= DESLOC_STATIC_MAX_POINTERS, M <= 8, and at most
- * DESLOC_STATIC_MAX_CHUNKS chunks of desloc_chunk_elems() elements (every tensor starts a new
- * chunk) -- up to 64 Mi parameters when tensors are large.  Anything bigger returns
- * DESLOC_E_TOO_LARGE and does nothing.
+ * DESLOC_STATIC_MAX_CHUNKS chunks (the chunk length is the one a context would use for the
+ * same tensor list; every tensor starts a new chunk) -- up to 64 Mi parameters when tensors
+ * are large.  Anything bigger returns DESLOC_E_TOO_LARGE and does nothing.
  *
  * Arguments as for desloc_create() + desloc_step(): cfg, the host arrays x, u, v, grads of
  * M*num_tensors DEVICE pointers (v may be NULL for SGDM), the step t, eta_t, the ADOPT bound,
- * the device and the stream.  State is updated in place; nothing is remembered between calls,
- * so there are no counters.  The tables are built on the calling thread's stack (about 320 KB
- * of it) and copied to the device on `stream` ahead of the kernel.
+ * the device and the stream.  State is updated in place; there are no counters.  All argument
+ * checks happen before the first CUDA call, so a rejected call (NULL, range, invalid, too
+ * large) touches neither the device nor the array.
  *
- * The first call on each device looks up the device address of the scratch array
- * (cudaGetSymbolAddress, with that device current); make that first call before any stream
- * capture begins.  All calls on a device share the one array and it keeps the previous
- * call's tables: each call rewrites the part it uses, nothing in it needs to start at zero.
- * Two calls whose GPU work can overlap -- different streams without an ordering between them,
- * or two host threads -- race on the array and must be serialised by the caller; calls issued
- * one after the other on the same stream are safe.
+ * Set-up.  The first call on each device looks up the device address of the array
+ * (cudaGetSymbolAddress, with that device current).  With the CUDA runtime's lazy module
+ * loading that look-up is also the moment the runtime loads the module and reserves the
+ * array's 320 KB on that GPU: make the first call at start-up -- before a framework's pool has
+ * grown to fill the device, where it could fail with DESLOC_E_CUDA, and before any stream
+ * capture begins.  The address is remembered per device for the life of the process and does
+ * not survive a cudaDeviceReset().
+ *
+ * Uploads.  The library keeps a host copy of what it last wrote into the array.  A call
+ * uploads only the tables that differ from it (the chunk table depends on the tensor list
+ * alone, the four pointer tables on x, u, v, grads), from ordinary pageable host memory,
+ * ahead of the kernel on `stream`; such a copy may wait for work already enqueued on `stream`
+ * before it returns.  A loop that steps the same buffers every time uploads nothing after its
+ * first call and only enqueues the kernel.  Because those copies read host memory the library
+ * reuses, the call returns DESLOC_E_INVALID, enqueueing nothing, while `stream` is being
+ * captured.
+ *
+ * Sharing.  All calls on a device share the one array, and it keeps the previous call's
+ * tables: each call rewrites what it needs, nothing in it has to start at zero.  Host threads
+ * are serialised inside the call, but two calls whose GPU work can overlap -- different
+ * streams without an ordering between them -- race on the array and must be ordered by the
+ * caller; calls issued one after the other on the same stream are safe.
  */
 #define DESLOC_STATIC_MAX_POINTERS 2048
 #define DESLOC_STATIC_MAX_CHUNKS 16384

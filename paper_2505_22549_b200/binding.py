@@ -12,8 +12,7 @@ import os
 from typing import Optional, Sequence
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-# DESLOC_LIBRARY selects another build of the same library (e.g. a tuning variant).
-LIB_PATH = os.environ.get("DESLOC_LIBRARY") or os.path.join(_HERE, "lib", "libdesloc.so")
+LIB_PATH = os.path.join(_HERE, "lib", "libdesloc.so")
 
 DESLOC_ADAM, DESLOC_ADOPT, DESLOC_SGDM = 0, 1, 2
 DESLOC_F32, DESLOC_BF16 = 0, 1
@@ -99,8 +98,14 @@ _lib.desloc_get_counters.restype = ctypes.c_int
 _lib.desloc_get_counters.argtypes = [_P, ctypes.POINTER(ctypes.c_int64)]
 _lib.desloc_get_launch_count.restype = ctypes.c_int64
 _lib.desloc_get_launch_count.argtypes = [_P]
-_lib.desloc_set_launch_shape.restype = ctypes.c_int
-_lib.desloc_set_launch_shape.argtypes = [_P, ctypes.c_int32]
+_lib.desloc_step_diag.restype = ctypes.c_int
+_lib.desloc_step_diag.argtypes = [_P, ctypes.c_int64, ctypes.c_float, ctypes.c_float,
+                                  ctypes.c_float, _PP, _P, ctypes.POINTER(ctypes.c_uint32)]
+_lib.desloc_get_diag_norms.restype = ctypes.c_int
+_lib.desloc_get_diag_norms.argtypes = [_P, ctypes.POINTER(ctypes.c_float),
+                                       ctypes.POINTER(ctypes.c_float), _P]
+_lib.desloc_testing_set_max_blocks.restype = ctypes.c_int
+_lib.desloc_testing_set_max_blocks.argtypes = [_P, ctypes.c_int64]
 _lib.desloc_plan_chunks.restype = ctypes.c_int64
 _lib.desloc_plan_chunks.argtypes = [ctypes.POINTER(ctypes.c_int64), ctypes.c_int32,
                                     ctypes.c_int64, ctypes.POINTER(ctypes.c_int64),
@@ -220,6 +225,33 @@ def desloc_step_normclip(ctx: int, t: int, lr_t: float, clip_bound_t: float, max
     return int(mask.value)
 
 
+def desloc_step_diag(ctx: int, t: int, lr_t: float, clip_bound_t: float, max_norm: float,
+                     grads, stream: int = 0) -> int:
+    """One step that also accumulates the gradient / parameter / update norms (max_norm > 0 adds
+    norm-based clipping in front, 0 = off); returns the sync mask."""
+    g = grads if isinstance(grads, ctypes.Array) else _ptr_array(grads)
+    mask = ctypes.c_uint32(0)
+    rc = _lib.desloc_step_diag(ctx, int(t), float(lr_t), float(clip_bound_t), float(max_norm), g,
+                               stream or None, ctypes.byref(mask))
+    if rc != DESLOC_OK:
+        raise DeslocError(rc, "desloc_step_diag", _lib.desloc_last_cuda_error(ctx))
+    return int(mask.value)
+
+
+def desloc_get_diag_norms(ctx: int, M: int, num_tensors: int, stream: int = 0):
+    """Norms of the latest desloc_step_diag: (per_tensor, total) as nested lists indexed
+    [kind][worker][tensor] and [kind][worker]; kind 0 = gradient, 1 = parameters, 2 = update."""
+    per = (ctypes.c_float * (3 * M * num_tensors))()
+    tot = (ctypes.c_float * (3 * M))()
+    rc = _lib.desloc_get_diag_norms(ctx, per, tot, stream or None)
+    if rc != DESLOC_OK:
+        raise DeslocError(rc, "desloc_get_diag_norms", _lib.desloc_last_cuda_error(ctx))
+    per_l = [[[per[(k * M + m) * num_tensors + j] for j in range(num_tensors)] for m in range(M)]
+             for k in range(3)]
+    tot_l = [[tot[k * M + m] for m in range(M)] for k in range(3)]
+    return per_l, tot_l
+
+
 def desloc_get_grad_norms(ctx: int, M: int, stream: int = 0):
     """(norms, clip factors) of the latest desloc_step_normclip as two lists of M floats."""
     norms, scales = (ctypes.c_float * M)(), (ctypes.c_float * M)()
@@ -264,10 +296,11 @@ def desloc_get_launch_count(ctx: int) -> int:
     return int(_lib.desloc_get_launch_count(ctx))
 
 
-def desloc_set_launch_shape(ctx: int, ctas_per_sm: int) -> None:
-    rc = _lib.desloc_set_launch_shape(ctx, int(ctas_per_sm))
+def desloc_testing_set_max_blocks(ctx: int, max_blocks: int) -> None:
+    """Test hook (include/desloc_testing.h): cap the step kernels' grid so that blocks stride."""
+    rc = _lib.desloc_testing_set_max_blocks(ctx, int(max_blocks))
     if rc != DESLOC_OK:
-        raise DeslocError(rc, "desloc_set_launch_shape")
+        raise DeslocError(rc, "desloc_testing_set_max_blocks")
 
 
 def desloc_chunk_elems() -> int:

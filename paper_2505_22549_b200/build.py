@@ -49,22 +49,10 @@ def _fingerprint(src: str) -> str:
     return h.hexdigest()
 
 
-def build(force: bool = False, verbose: bool = False, extra_flags=(), out: str | None = None,
-          obj_dir: str | None = None) -> str:
+def build(force: bool = False, verbose: bool = False) -> str:
     """Compile every translation unit (in parallel) and link the shared library.
-
-    extra_flags / out / obj_dir build a tuning variant (e.g. -DDESLOC_MINB_LARGE_M=3) into
-    another file without touching the default library."""
-    global OBJ, LIB
-    saved = (OBJ, LIB)
-    if obj_dir:
-        OBJ = obj_dir
-    if out:
-        LIB = out
-    try:
-        return _build(force, verbose, list(extra_flags))
-    finally:
-        OBJ, LIB = saved
+    verbose passes -Xptxas -v and prints the compiler's register / spill report to stderr."""
+    return _build(force, verbose, [])
 
 
 def _build(force: bool, verbose: bool, extra_flags) -> str:
@@ -96,7 +84,7 @@ def _build(force: bool, verbose: bool, extra_flags) -> str:
     if not any(changed for _, changed in results) and os.path.exists(LIB):
         return LIB
     tmp = LIB + f".tmp{os.getpid()}"
-    cmd = [nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + objs
+    cmd = [nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + objs + ["-ldl"]
     r = subprocess.run(cmd, capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")

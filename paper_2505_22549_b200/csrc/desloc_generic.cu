@@ -1,31 +1,58 @@
 // DES-LOC step for worker counts beyond the register-resident kernels (M > MAX_MT) on steps
-// that average something.  Same update (update_coord with one worker at a time), runtime M and
-// mask.  Worker sums are accumulated in fp64 in the order m = 0..M-1, which is exact for equal
+// that average something.  Same update as desloc_step_kernel, runtime M, compile-time mask.
+// Worker sums are accumulated in fp64 in the order m = 0..M-1, which is exact for equal
 // replicas and matches a sequential reference to rounding.
 //
-// Pre-average ordering: pass 1 reads only the arrays to be averaged and forms their means;
-// pass 2 reads the remaining arrays and updates every worker -- each array is still read once
-// (ADOPT re-reads its own v on v-sync steps for the normaliser).  Post-average ordering needs
-// the updated states of all workers before any parameter step, so it stores the local u, v
-// first and revisits them (the revisit is served from cache).
+// A block takes one chunk and first puts the chunk-relative pointers of all M workers into
+// shared memory, so that the per-position loops read them as broadcasts instead of chasing the
+// pointer tables in global memory.  Per position (4 elements per thread):
+//   pre-average   the arrays to be averaged are summed one array at a time, eight workers'
+//                 loads in flight; then the workers are updated in batches sized to the
+//                 register budget, loading only what was not averaged (ADOPT also its own v).
+//                 Each array is read once and written once.
+//   post-average  phase A updates the states batch by batch, sums the ones to be averaged and
+//                 stores the others; the parameter step runs in phase A when d_t uses only the
+//                 worker's own states, otherwise in phase B once the means are known.  Only
+//                 when Adam averages exactly one of u, v does phase B re-read the other one
+//                 (just written, so it is served from cache).
 #include "desloc_kernels.cuh"
 
 namespace desloc {
 
-struct Ptrs {
-    char *x, *u, *v;
-    const char *g;
-};
+namespace {
 
-template <int OPT, typename GT>
-__device__ __forceinline__ Ptrs worker_ptrs(const StepArgs &a, const Chunk &ch, int m) {
-    const long long idx = static_cast<long long>(m) * a.nt + ch.tensor;
-    Ptrs p;
-    p.x = reinterpret_cast<char *>(a.x[idx]) + ch.start * 4;
-    p.u = reinterpret_cast<char *>(a.u[idx]) + ch.start * 4;
-    p.v = (OPT != OPT_SGDM) ? reinterpret_cast<char *>(a.v[idx]) + ch.start * 4 : nullptr;
-    p.g = reinterpret_cast<const char *>(grad_ptr(a, idx)) + ch.start * static_cast<long long>(sizeof(GT));
-    return p;
+constexpr int GEN_MAX_M = 256;    // worker pointers staged per chunk (= the context's limit)
+constexpr int MEAN_BATCH = 4;     // workers whose loads are in flight while an array is summed
+
+// Workers per batch of the update loops: what fits in `budget` registers, at most four.
+__host__ __device__ constexpr int gen_batch(int per_worker, int budget) {
+    const int b = budget / per_worker;
+    return b < 1 ? 1 : (b > 4 ? 4 : b);
+}
+
+template <int VEC>
+__device__ __forceinline__ FV<VEC> mean_f64(char *const *bases, int M, long long e, bool active) {
+    double acc[VEC];
+#pragma unroll
+    for (int c = 0; c < VEC; ++c) acc[c] = 0.0;
+#pragma unroll 1
+    for (int m0 = 0; m0 < M; m0 += MEAN_BATCH) {
+        FV<VEC> b[MEAN_BATCH];
+#pragma unroll
+        for (int j = 0; j < MEAN_BATCH; ++j)
+            if (active && m0 + j < M) b[j] = ld_f32<VEC>(bases[m0 + j], e);
+#pragma unroll
+        for (int j = 0; j < MEAN_BATCH; ++j) {
+            if (active && m0 + j < M) {
+#pragma unroll
+                for (int c = 0; c < VEC; ++c) acc[c] += static_cast<double>(b[j].a[c]);
+            }
+        }
+    }
+    FV<VEC> r;
+#pragma unroll
+    for (int c = 0; c < VEC; ++c) r.a[c] = static_cast<float>(acc[c] / static_cast<double>(M));
+    return r;
 }
 
 template <int VEC>
@@ -42,229 +69,315 @@ __device__ __forceinline__ FV<VEC> acc_mean(const double (&acc)[VEC], int M) {
     return r;
 }
 
-// default-cached loads here: the second visit of an address should hit in L1/L2
-template <int VEC>
-__device__ __forceinline__ FV<VEC> ld_plain(const char *base, long long e) {
-    FV<VEC> r;
-    if constexpr (VEC == 4) {
-        const float4 t = *(reinterpret_cast<const float4 *>(base) + (e >> 2));
-        r.a[0] = t.x; r.a[1] = t.y; r.a[2] = t.z; r.a[3] = t.w;
-    } else {
-        r.a[0] = *(reinterpret_cast<const float *>(base) + e);
+// Diagnostics with a runtime worker count: a warp reduces each (kind, worker) value at once
+// and lane 0 adds it to the warp's own row of shared memory, in position order.
+template <bool DIAG>
+struct WarpDiag {
+    float *rows;  // [BLOCK_THREADS / 32][DIAG_KINDS][GEN_MAX_M]
+    __device__ __forceinline__ void add(int kind, int m, float v) const {
+        if constexpr (DIAG) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) v += __shfl_down_sync(0xffffffffu, v, off);
+            if ((threadIdx.x & 31) == 0)
+                rows[((threadIdx.x >> 5) * DIAG_KINDS + kind) * GEN_MAX_M + m] += v;
+        }
     }
-    return r;
-}
+    // the same value for every worker (a synced x): one reduction, M additions by lane 0
+    __device__ __forceinline__ void add_all(int kind, int M, float v) const {
+        if constexpr (DIAG) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) v += __shfl_down_sync(0xffffffffu, v, off);
+            if ((threadIdx.x & 31) == 0) {
+                float *row = rows + ((threadIdx.x >> 5) * DIAG_KINDS + kind) * GEN_MAX_M;
+                for (int m = 0; m < M; ++m) row[m] += v;
+            }
+        }
+    }
+};
 
-// CMASK >= 0: the sync mask is a compile-time constant (pre-average instantiations, so that
-// arrays that are not averaged cost no registers); CMASK < 0: taken from mask_rt.
-template <int OPT, typename GT, bool POST, int CMASK, int VEC>
-__device__ __forceinline__ void generic_position(const StepArgs &a, const Chunk &ch, int mask_rt,
-                                                 long long e) {
-    const int mask = CMASK >= 0 ? CMASK : mask_rt;
+// One position (VEC elements) of all M workers.  `active` is false for the lanes a DIAG warp
+// carries past the end of the chunk: they touch no memory and contribute zeros to the sums.
+template <int OPT, typename GT, bool POST, int MASK, int VEC, bool DIAG>
+__device__ __forceinline__ void generic_position(const StepArgs &a, char *const (*sp)[GEN_MAX_M],
+                                                 const float *sscale, long long e, bool active,
+                                                 const WarpDiag<DIAG> &wd) {
     const int M = a.M;
-    const bool sx = mask & SYNC_X, su = mask & SYNC_U, sv = (OPT != OPT_SGDM) && (mask & SYNC_V);
+    constexpr bool SX = MASK & SYNC_X, SU = MASK & SYNC_U;
+    constexpr bool SV = (OPT != OPT_SGDM) && (MASK & SYNC_V);
     if constexpr (!POST) {
-        double ax[VEC] = {}, au[VEC] = {}, av[VEC] = {};
-        // several workers at a time so that their pointer and data loads overlap (four when one
-        // array is averaged, two for two, one for three: more would spill under the register
-        // cap); the sums still run in the order m = 0..M-1
-        constexpr int NSYNC = CMASK < 0 ? 3 : ((CMASK & 1) + ((CMASK >> 1) & 1) + ((CMASK >> 2) & 1));
-        constexpr int NB = NSYNC <= 1 ? 4 : (NSYNC == 2 ? 2 : 1);
+        FV<VEC> xb{}, ub{}, vb{};
+        if constexpr (SX) xb = mean_f64<VEC>(sp[0], M, e, active);
+        if constexpr (SU) ub = mean_f64<VEC>(sp[1], M, e, active);
+        if constexpr (SV) vb = mean_f64<VEC>(sp[2], M, e, active);
+        constexpr bool NEED_V = OPT != OPT_SGDM && (!SV || OPT == OPT_ADOPT);
+        constexpr int B = gen_batch(worker_regs<OPT, GT>(!SX, !SU, NEED_V), 48);
 #pragma unroll 1
-        for (int m0 = 0; m0 < M; m0 += NB) {
-            FV<VEC> bx[NB], bu[NB], bv[NB];
+        for (int m0 = 0; m0 < M; m0 += B) {
+            FV<VEC> G[B], X[B], U[B], V[B];
 #pragma unroll
-            for (int j = 0; j < NB; ++j) {
-                if (m0 + j < M) {
-                    const Ptrs p = worker_ptrs<OPT, GT>(a, ch, m0 + j);
-                    if (sx) bx[j] = ld_plain<VEC>(p.x, e);
-                    if (su) bu[j] = ld_plain<VEC>(p.u, e);
-                    if (sv) bv[j] = ld_plain<VEC>(p.v, e);
+            for (int b = 0; b < B; ++b) {
+                if (active && m0 + b < M) {
+                    G[b] = ld_grad<VEC, GT>(sp[3][m0 + b], e);
+                    if constexpr (!SX) X[b] = ld_f32<VEC>(sp[0][m0 + b], e);
+                    if constexpr (!SU) U[b] = ld_f32<VEC>(sp[1][m0 + b], e);
+                    if constexpr (NEED_V) V[b] = ld_f32<VEC>(sp[2][m0 + b], e);
                 }
             }
 #pragma unroll
-            for (int j = 0; j < NB; ++j) {
-                if (m0 + j < M) {
-                    if (sx) acc_add<VEC>(ax, bx[j]);
-                    if (su) acc_add<VEC>(au, bu[j]);
-                    if (sv) acc_add<VEC>(av, bv[j]);
+            for (int b = 0; b < B; ++b) {
+                if (m0 + b < M) {
+                    float gg = 0.f, dd = 0.f, xx = 0.f;
+                    if (active) {
+                        gg = sum_sq<VEC>(G[b]);
+                        const float sc = sscale[m0 + b];
+                        FV<VEC> D;
+#pragma unroll
+                        for (int c = 0; c < VEC; ++c) {
+                            const float up = SU ? ub.a[c] : U[b].a[c];
+                            const float vown = NEED_V ? V[b].a[c] : 0.f;
+                            const float vp = SV ? vb.a[c] : vown;
+                            const float xp = SX ? xb.a[c] : X[b].a[c];
+                            float un, vn;
+                            state_update<OPT>(a, G[b].a[c] * sc, up, vp, vown, un, vn);
+                            D.a[c] = direction<OPT>(a, un, vn);
+                            X[b].a[c] = apply_step(a, xp, D.a[c]);
+                            U[b].a[c] = un;
+                            V[b].a[c] = vn;
+                        }
+                        dd = sum_sq<VEC>(D);
+                        xx = sum_sq<VEC>(X[b]);
+                        st_f32<VEC>(sp[0][m0 + b], e, X[b]);
+                        st_f32<VEC>(sp[1][m0 + b], e, U[b]);
+                        if constexpr (OPT != OPT_SGDM) st_f32<VEC>(sp[2][m0 + b], e, V[b]);
+                    }
+                    wd.add(DIAG_G, m0 + b, gg);
+                    wd.add(DIAG_D, m0 + b, dd);
+                    wd.add(DIAG_X, m0 + b, xx);
                 }
             }
-        }
-        const FV<VEC> xb = acc_mean<VEC>(ax, M), ub = acc_mean<VEC>(au, M), vb = acc_mean<VEC>(av, M);
-        for (int m = 0; m < M; ++m) {
-            const Ptrs p = worker_ptrs<OPT, GT>(a, ch, m);
-            FV<VEC> G = ld_grad<VEC, GT>(p.g, e);
-            if (a.gscale) {
-                const float sc = a.gscale[m];
-#pragma unroll
-                for (int c = 0; c < VEC; ++c) G.a[c] *= sc;
-            }
-            FV<VEC> X = sx ? xb : ld_f32<VEC>(p.x, e);
-            FV<VEC> U = su ? ub : ld_f32<VEC>(p.u, e);
-            FV<VEC> V{}, Vown{};
-            if constexpr (OPT != OPT_SGDM) {
-                if (OPT == OPT_ADOPT || !sv) Vown = ld_plain<VEC>(p.v, e);
-                V = sv ? vb : Vown;
-            }
-#pragma unroll
-            for (int c = 0; c < VEC; ++c) {
-                // one worker at a time: hand the averaged values in as that worker's "previous"
-                // state; ADOPT's normaliser must see the worker's own v, so split it out.
-                float g1[1] = {G.a[c]}, x1[1] = {X.a[c]}, u1[1] = {U.a[c]}, v1[1] = {V.a[c]};
-                if constexpr (OPT == OPT_ADOPT) {
-                    const float gh = fminf(fmaxf(g1[0], -a.rho), a.rho);
-                    const float vn = fmaf(a.b2, v1[0], (a.omb2 * gh) * gh);
-                    float r = gh / fmaxf(sqrtf(Vown.a[c]), a.eps);
-                    r = fminf(fmaxf(r, -a.cbound), a.cbound);
-                    const float un = fmaf(a.b1, u1[0], a.omb1 * r);
-                    const float d = a.lr * un;
-                    x1[0] = x1[0] - fmaf(a.lrwd, x1[0], d);
-                    u1[0] = un;
-                    v1[0] = vn;
-                } else {
-                    update_coord<OPT, 0, 1, false>(a, g1, x1, u1, v1);
-                }
-                X.a[c] = x1[0]; U.a[c] = u1[0]; V.a[c] = v1[0];
-            }
-            st_f32<VEC>(p.x, e, X);
-            st_f32<VEC>(p.u, e, U);
-            if constexpr (OPT != OPT_SGDM) st_f32<VEC>(p.v, e, V);
         }
     } else {
-        // pass A: local state updates, stored; sums of the ones to be averaged
-        double au[VEC] = {}, av[VEC] = {}, ax[VEC] = {};
-        for (int m = 0; m < M; ++m) {
-            const Ptrs p = worker_ptrs<OPT, GT>(a, ch, m);
-            FV<VEC> G = ld_grad<VEC, GT>(p.g, e);
-            if (a.gscale) {
-                const float sc = a.gscale[m];
+        using P = PostPlan<OPT, MASK>;
+        double au[VEC], av[VEC], ax[VEC];
 #pragma unroll
-                for (int c = 0; c < VEC; ++c) G.a[c] *= sc;
-            }
-            FV<VEC> U = ld_f32<VEC>(p.u, e), V{};
-            if constexpr (OPT != OPT_SGDM) V = ld_f32<VEC>(p.v, e);
+        for (int c = 0; c < VEC; ++c) au[c] = av[c] = ax[c] = 0.0;
+        constexpr int BA = gen_batch(worker_regs<OPT, GT>(!P::D_NEEDS_MEAN, true, OPT != OPT_SGDM), 48);
+        // phase A: states (and x where d_t needs no mean)
+#pragma unroll 1
+        for (int m0 = 0; m0 < M; m0 += BA) {
+            FV<VEC> G[BA], U[BA], V[BA], X[BA];
 #pragma unroll
-            for (int c = 0; c < VEC; ++c) {
-                const float gh = fminf(fmaxf(G.a[c], -a.rho), a.rho);
-                if constexpr (OPT == OPT_ADAM) {
-                    U.a[c] = fmaf(a.b1, U.a[c], a.omb1 * gh);
-                    V.a[c] = fmaf(a.b2, V.a[c], (a.omb2 * gh) * gh);
-                } else if constexpr (OPT == OPT_ADOPT) {
-                    float r = gh / fmaxf(sqrtf(V.a[c]), a.eps);
-                    r = fminf(fmaxf(r, -a.cbound), a.cbound);
-                    U.a[c] = fmaf(a.b1, U.a[c], a.omb1 * r);
-                    V.a[c] = fmaf(a.b2, V.a[c], (a.omb2 * gh) * gh);
-                } else {
-                    U.a[c] = fmaf(a.b1, U.a[c], a.omb1 * gh);
+            for (int b = 0; b < BA; ++b) {
+                if (active && m0 + b < M) {
+                    G[b] = ld_grad<VEC, GT>(sp[3][m0 + b], e);
+                    U[b] = ld_f32<VEC>(sp[1][m0 + b], e);
+                    if constexpr (OPT != OPT_SGDM) V[b] = ld_f32<VEC>(sp[2][m0 + b], e);
+                    if constexpr (!P::D_NEEDS_MEAN) X[b] = ld_f32<VEC>(sp[0][m0 + b], e);
                 }
             }
-            if (su) acc_add<VEC>(au, U);
-            if (sv) acc_add<VEC>(av, V);
-            // plain stores: pass B reads these back
-            if constexpr (VEC == 4) {
-                *(reinterpret_cast<float4 *>(p.u) + (e >> 2)) = make_float4(U.a[0], U.a[1], U.a[2], U.a[3]);
-                if constexpr (OPT != OPT_SGDM)
-                    *(reinterpret_cast<float4 *>(p.v) + (e >> 2)) = make_float4(V.a[0], V.a[1], V.a[2], V.a[3]);
-            } else {
-                *(reinterpret_cast<float *>(p.u) + e) = U.a[0];
-                if constexpr (OPT != OPT_SGDM) *(reinterpret_cast<float *>(p.v) + e) = V.a[0];
-            }
-        }
-        const FV<VEC> ub = acc_mean<VEC>(au, M), vb = acc_mean<VEC>(av, M);
-        // pass B: parameter step with the (possibly averaged) new states
-        for (int m = 0; m < M; ++m) {
-            const Ptrs p = worker_ptrs<OPT, GT>(a, ch, m);
-            FV<VEC> X = ld_f32<VEC>(p.x, e);
-            FV<VEC> U = su ? ub : ld_plain<VEC>(p.u, e), V{};
-            if constexpr (OPT == OPT_ADAM) V = sv ? vb : ld_plain<VEC>(p.v, e);
 #pragma unroll
-            for (int c = 0; c < VEC; ++c) {
-                float d;
-                if constexpr (OPT == OPT_ADAM)
-                    d = (a.lr * U.a[c]) / sqrtf(V.a[c] + a.lam2);
-                else
-                    d = a.lr * U.a[c];
-                X.a[c] = X.a[c] - fmaf(a.lrwd, X.a[c], d);
+            for (int b = 0; b < BA; ++b) {
+                if (m0 + b < M) {
+                    float gg = 0.f, dd = 0.f, xx = 0.f;
+                    if (active) {
+                        gg = sum_sq<VEC>(G[b]);
+                        const float sc = sscale[m0 + b];
+                        FV<VEC> D;
+#pragma unroll
+                        for (int c = 0; c < VEC; ++c) {
+                            const float vown = OPT != OPT_SGDM ? V[b].a[c] : 0.f;
+                            float un, vn;
+                            state_update<OPT>(a, G[b].a[c] * sc, U[b].a[c], vown, vown, un, vn);
+                            U[b].a[c] = un;
+                            V[b].a[c] = vn;
+                            if constexpr (!P::D_NEEDS_MEAN) {
+                                D.a[c] = direction<OPT>(a, un, vn);
+                                X[b].a[c] = apply_step(a, X[b].a[c], D.a[c]);
+                            }
+                        }
+                        // a state that is not averaged has its final value now (phase B re-reads
+                        // it where Adam needs it per worker)
+                        if constexpr (!P::SU) st_f32<VEC>(sp[1][m0 + b], e, U[b]);
+                        if constexpr (OPT != OPT_SGDM && !P::SV) st_f32<VEC>(sp[2][m0 + b], e, V[b]);
+                        if constexpr (P::SU) acc_add<VEC>(au, U[b]);
+                        if constexpr (P::SV) acc_add<VEC>(av, V[b]);
+                        if constexpr (!P::D_NEEDS_MEAN) {
+                            dd = sum_sq<VEC>(D);
+                            if constexpr (P::SX) {
+                                acc_add<VEC>(ax, X[b]);
+                            } else {
+                                xx = sum_sq<VEC>(X[b]);
+                                st_f32<VEC>(sp[0][m0 + b], e, X[b]);
+                            }
+                        }
+                    }
+                    wd.add(DIAG_G, m0 + b, gg);
+                    if constexpr (!P::D_NEEDS_MEAN) {
+                        wd.add(DIAG_D, m0 + b, dd);
+                        if constexpr (!P::SX) wd.add(DIAG_X, m0 + b, xx);
+                    }
+                }
             }
-            if (sx) acc_add<VEC>(ax, X); else st_f32<VEC>(p.x, e, X);
-            if (su) st_f32<VEC>(p.u, e, ub);
-            if constexpr (OPT != OPT_SGDM) if (sv) st_f32<VEC>(p.v, e, vb);
         }
-        if (sx) {
-            const FV<VEC> xb = acc_mean<VEC>(ax, M);
-            for (int m = 0; m < M; ++m) {
-                const Ptrs p = worker_ptrs<OPT, GT>(a, ch, m);
-                st_f32<VEC>(p.x, e, xb);
+        const FV<VEC> mu = acc_mean<VEC>(au, M), mv = acc_mean<VEC>(av, M);
+        if constexpr (P::D_NEEDS_MEAN) {
+            // phase B: parameter step with the averaged states
+            constexpr int BB = gen_batch(4 + ((P::KEEP_U || P::KEEP_V) ? 4 : 0), 48);
+#pragma unroll 1
+            for (int m0 = 0; m0 < M; m0 += BB) {
+                FV<VEC> X[BB], K[BB];
+#pragma unroll
+                for (int b = 0; b < BB; ++b) {
+                    if (active && m0 + b < M) {
+                        X[b] = ld_f32<VEC>(sp[0][m0 + b], e);
+                        if constexpr (P::KEEP_U) K[b] = ld_f32<VEC>(sp[1][m0 + b], e);
+                        if constexpr (P::KEEP_V) K[b] = ld_f32<VEC>(sp[2][m0 + b], e);
+                    }
+                }
+#pragma unroll
+                for (int b = 0; b < BB; ++b) {
+                    if (m0 + b < M) {
+                        float dd = 0.f, xx = 0.f;
+                        if (active) {
+                            FV<VEC> D;
+#pragma unroll
+                            for (int c = 0; c < VEC; ++c) {
+                                const float un = P::SU ? mu.a[c] : K[b].a[c];
+                                const float vn = P::SV ? mv.a[c] : (P::KEEP_V ? K[b].a[c] : 0.f);
+                                D.a[c] = direction<OPT>(a, un, vn);
+                                X[b].a[c] = apply_step(a, X[b].a[c], D.a[c]);
+                            }
+                            dd = sum_sq<VEC>(D);
+                            if constexpr (P::SX) {
+                                acc_add<VEC>(ax, X[b]);
+                            } else {
+                                xx = sum_sq<VEC>(X[b]);
+                                st_f32<VEC>(sp[0][m0 + b], e, X[b]);
+                            }
+                            if constexpr (P::SU) st_f32<VEC>(sp[1][m0 + b], e, mu);
+                            if constexpr (P::SV) st_f32<VEC>(sp[2][m0 + b], e, mv);
+                        }
+                        wd.add(DIAG_D, m0 + b, dd);
+                        if constexpr (!P::SX) wd.add(DIAG_X, m0 + b, xx);
+                    }
+                }
             }
+        }
+        if constexpr (P::SX || (!P::D_NEEDS_MEAN && P::SV)) {
+            const FV<VEC> mx = acc_mean<VEC>(ax, M);
+            const float xx = (P::SX && active) ? sum_sq<VEC>(mx) : 0.f;
+            if (active) {
+#pragma unroll 1
+                for (int m = 0; m < M; ++m) {
+                    if constexpr (P::SX) st_f32<VEC>(sp[0][m], e, mx);
+                    if constexpr (!P::D_NEEDS_MEAN && P::SV) st_f32<VEC>(sp[2][m], e, mv);
+                }
+            }
+            if constexpr (P::SX) wd.add_all(DIAG_X, M, xx);
         }
     }
 }
 
-template <int OPT, typename GT, bool POST, int CMASK>
-__global__ void __launch_bounds__(BLOCK_THREADS, 4)
-desloc_step_generic_kernel(const __grid_constant__ StepArgs a, const int mask) {
-    __shared__ int s_mis;
+template <int OPT, typename GT, bool POST, int MASK, bool DIAG>
+__global__ void __launch_bounds__(BLOCK_THREADS, 2)
+desloc_step_generic_kernel(const __grid_constant__ StepArgs a) {
+    __shared__ char *sp[4][GEN_MAX_M];
+    __shared__ float sscale[GEN_MAX_M];
+    __shared__ float srows[DIAG ? (BLOCK_THREADS / 32) * DIAG_KINDS * GEN_MAX_M : 1];
+    const WarpDiag<DIAG> wd{srows};
     const int tid = threadIdx.x;
-    for (long long c = blockIdx.x; c < a.nchunks; c += gridDim.x) {
+    const int lane = tid & 31;
+    // exactly one chunk per block (this kernel does not stride: with a chunk loop around the
+    // same body the compiler needs spill slots)
+    const long long c = blockIdx.x;
+    if (c < a.nchunks) {
         const Chunk ch = a.chunks[c];
-        if (tid == 0) s_mis = 0;
-        __syncthreads();
-        // alignment of every worker's four pointers decides vector vs scalar for the chunk
         int mis = 0;
         for (int m = tid; m < a.M; m += BLOCK_THREADS) {
-            const Ptrs p = worker_ptrs<OPT, GT>(a, ch, m);
-            mis |= (reinterpret_cast<uintptr_t>(p.x) | reinterpret_cast<uintptr_t>(p.u)) & 15u;
-            if (OPT != OPT_SGDM) mis |= reinterpret_cast<uintptr_t>(p.v) & 15u;
-            mis |= reinterpret_cast<uintptr_t>(p.g) & (sizeof(GT) == 2 ? 7u : 15u);
+            const long long idx = static_cast<long long>(m) * a.nt + ch.tensor;
+            char *px = reinterpret_cast<char *>(a.x[idx]) + ch.start * 4;
+            char *pu = reinterpret_cast<char *>(a.u[idx]) + ch.start * 4;
+            char *pv = (OPT != OPT_SGDM) ? reinterpret_cast<char *>(a.v[idx]) + ch.start * 4 : nullptr;
+            char *pg = const_cast<char *>(reinterpret_cast<const char *>(grad_ptr(a, idx))) +
+                       ch.start * static_cast<long long>(sizeof(GT));
+            sp[0][m] = px; sp[1][m] = pu; sp[2][m] = pv; sp[3][m] = pg;
+            sscale[m] = a.gscale ? a.gscale[m] : 1.f;
+            mis |= (reinterpret_cast<uintptr_t>(px) | reinterpret_cast<uintptr_t>(pu) |
+                    reinterpret_cast<uintptr_t>(pv)) & 15u;
+            mis |= reinterpret_cast<uintptr_t>(pg) & (sizeof(GT) == 2 ? 7u : 15u);
         }
-        if (mis) atomicOr(&s_mis, 1);
-        __syncthreads();
-        const bool scalar_path = s_mis != 0;
-        __syncthreads();
+        if constexpr (DIAG) {
+            for (int j = tid; j < (BLOCK_THREADS / 32) * DIAG_KINDS * GEN_MAX_M; j += BLOCK_THREADS)
+                srows[j] = 0.f;
+        }
+        const bool scalar_path = __syncthreads_or(mis) != 0;
+        // DIAG warps run whole: lanes past the end take part in the shuffles with zeros
         if (!scalar_path) {
             const int n4 = ch.count >> 2;
-            for (int p0 = tid; p0 < n4; p0 += BLOCK_THREADS)
-                generic_position<OPT, GT, POST, CMASK, 4>(a, ch, mask, static_cast<long long>(p0) * 4);
+            for (int p = tid; DIAG ? (p - lane < n4) : (p < n4); p += BLOCK_THREADS)
+                generic_position<OPT, GT, POST, MASK, 4, DIAG>(a, sp, sscale, static_cast<long long>(p) * 4,
+                                                              p < n4, wd);
             const int rem = ch.count & 3;
-            if (tid < rem) generic_position<OPT, GT, POST, CMASK, 1>(a, ch, mask, (n4 << 2) + tid);
+            if (DIAG ? (tid < 32 && rem > 0) : (tid < rem))
+                generic_position<OPT, GT, POST, MASK, 1, DIAG>(a, sp, sscale, (n4 << 2) + tid, tid < rem, wd);
         } else {
-            for (int e = tid; e < ch.count; e += BLOCK_THREADS)
-                generic_position<OPT, GT, POST, CMASK, 1>(a, ch, mask, e);
+            for (int e = tid; DIAG ? (e - lane < ch.count) : (e < ch.count); e += BLOCK_THREADS)
+                generic_position<OPT, GT, POST, MASK, 1, DIAG>(a, sp, sscale, e, e < ch.count, wd);
+        }
+        if constexpr (DIAG) {
+            __syncthreads();
+            for (int j = tid; j < DIAG_KINDS * a.M; j += BLOCK_THREADS) {
+                const int kind = j / a.M, m = j - kind * a.M;
+                float total = 0.f;
+#pragma unroll
+                for (int w = 0; w < BLOCK_THREADS / 32; ++w)
+                    total += srows[(w * DIAG_KINDS + kind) * GEN_MAX_M + m];
+                a.diag[(static_cast<long long>(kind) * a.M + m) * a.diag_stride + a.diag_chunk0 + c] = total;
+            }
         }
     }
 }
 
-template <int OPT, typename GT, bool POST, int CMASK>
-static const void *generic_ptr() {
-    return reinterpret_cast<const void *>(&desloc_step_generic_kernel<OPT, GT, POST, CMASK>);
+template <int OPT, typename GT, bool POST, bool DIAG, int MASK>
+const void *generic_ptr() {
+    return reinterpret_cast<const void *>(&desloc_step_generic_kernel<OPT, GT, POST, MASK, DIAG>);
 }
 
-template <int OPT, typename GT>
-static const void *pick_generic(bool post, int mask) {
-    if (post) return generic_ptr<OPT, GT, true, -1>();
+template <int OPT, typename GT, bool POST, bool DIAG>
+const void *pick_mask(int mask) {
     switch (mask) {
-        case 1: return generic_ptr<OPT, GT, false, 1>();
-        case 2: return generic_ptr<OPT, GT, false, 2>();
-        case 3: return generic_ptr<OPT, GT, false, 3>();
+        case 1: return generic_ptr<OPT, GT, POST, DIAG, 1>();
+        case 2: return generic_ptr<OPT, GT, POST, DIAG, 2>();
+        case 3: return generic_ptr<OPT, GT, POST, DIAG, 3>();
         default: break;
     }
     if constexpr (OPT != OPT_SGDM) {
         switch (mask) {
-            case 4: return generic_ptr<OPT, GT, false, 4>();
-            case 5: return generic_ptr<OPT, GT, false, 5>();
-            case 6: return generic_ptr<OPT, GT, false, 6>();
-            case 7: return generic_ptr<OPT, GT, false, 7>();
+            case 4: return generic_ptr<OPT, GT, POST, DIAG, 4>();
+            case 5: return generic_ptr<OPT, GT, POST, DIAG, 5>();
+            case 6: return generic_ptr<OPT, GT, POST, DIAG, 6>();
+            case 7: return generic_ptr<OPT, GT, POST, DIAG, 7>();
             default: break;
         }
     }
     return nullptr;
 }
 
-const void *lookup_generic_kernel(int opt, bool post, bool bf16, int mask) {
-    if (opt == OPT_ADAM) return bf16 ? pick_generic<OPT_ADAM, bf16_t>(post, mask) : pick_generic<OPT_ADAM, float>(post, mask);
-    if (opt == OPT_ADOPT) return bf16 ? pick_generic<OPT_ADOPT, bf16_t>(post, mask) : pick_generic<OPT_ADOPT, float>(post, mask);
-    if (opt == OPT_SGDM) return bf16 ? pick_generic<OPT_SGDM, bf16_t>(post, mask) : pick_generic<OPT_SGDM, float>(post, mask);
+template <int OPT, typename GT>
+const void *pick_generic(bool post, int mask, bool diag) {
+    if (post) return diag ? pick_mask<OPT, GT, true, true>(mask) : pick_mask<OPT, GT, true, false>(mask);
+    return diag ? pick_mask<OPT, GT, false, true>(mask) : pick_mask<OPT, GT, false, false>(mask);
+}
+
+}  // namespace
+
+const void *lookup_generic_kernel(int opt, bool post, bool bf16, int mask, bool diag) {
+    if (opt == OPT_ADAM)
+        return bf16 ? pick_generic<OPT_ADAM, bf16_t>(post, mask, diag) : pick_generic<OPT_ADAM, float>(post, mask, diag);
+    if (opt == OPT_ADOPT)
+        return bf16 ? pick_generic<OPT_ADOPT, bf16_t>(post, mask, diag) : pick_generic<OPT_ADOPT, float>(post, mask, diag);
+    if (opt == OPT_SGDM)
+        return bf16 ? pick_generic<OPT_SGDM, bf16_t>(post, mask, diag) : pick_generic<OPT_SGDM, float>(post, mask, diag);
     return nullptr;
 }
 

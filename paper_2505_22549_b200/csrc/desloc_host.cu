@@ -11,30 +11,39 @@
 #include <new>
 #include <vector>
 
-#include "../../include/desloc.h"
+#include "../../include/desloc_testing.h"
 #include "desloc_inst.cuh"
+#include "desloc_internal.cuh"
 #include "desloc_norms.cuh"
 
 namespace desloc {
 
-const void *lookup_step_kernel(int opt, bool post, bool bf16, int mt, int mask) {
-    if (mask == 0) {
-        // Local step: the same code for either ordering.  Up to MAX_MT workers it uses the
-        // all-workers-per-chunk instantiation (more bytes per block and per pointer set-up);
-        // beyond that, and for M = 1, workers are separate work items of the MT = 1 kernel.
-        const int m = (mt >= 2 && mt <= MAX_MT) ? mt : 1;
-        if (opt == OPT_ADAM) return lookup_adam_pre(bf16, m, 0);
-        if (opt == OPT_ADOPT) return lookup_adopt_pre(bf16, m, 0);
-        if (opt == OPT_SGDM) return lookup_sgdm_pre(bf16, m, 0);
-        return nullptr;
+const void *lookup_step_kernel(int opt, bool post, bool bf16, int mt, int mask, bool diag) {
+    // A local step (mask 0) is the same code for either ordering and lives in the pre-average
+    // units.  Up to MAX_MT workers it uses the all-workers-per-chunk instantiation (more bytes
+    // per block and per pointer set-up); beyond that, and for M = 1, workers are separate work
+    // items of the local kernel.
+    const bool pre = !post || mask == 0;
+    const int m = (mask == 0 && !(mt >= 2 && mt <= MAX_MT)) ? 1 : mt;
+    if (opt == OPT_ADAM) {
+        if (diag) return pre ? lookup_adam_pre_diag(bf16, m, mask) : lookup_adam_post_diag(bf16, m, mask);
+        return pre ? lookup_adam_pre(bf16, m, mask) : lookup_adam_post(bf16, m, mask);
     }
-    if (opt == OPT_ADAM) return post ? lookup_adam_post(bf16, mt, mask) : lookup_adam_pre(bf16, mt, mask);
-    if (opt == OPT_ADOPT) return post ? lookup_adopt_post(bf16, mt, mask) : lookup_adopt_pre(bf16, mt, mask);
-    if (opt == OPT_SGDM) return post ? lookup_sgdm_post(bf16, mt, mask) : lookup_sgdm_pre(bf16, mt, mask);
+    if (opt == OPT_ADOPT) {
+        if (diag) return pre ? lookup_adopt_pre_diag(bf16, m, mask) : lookup_adopt_post_diag(bf16, m, mask);
+        return pre ? lookup_adopt_pre(bf16, m, mask) : lookup_adopt_post(bf16, m, mask);
+    }
+    if (opt == OPT_SGDM) {
+        if (diag) return pre ? lookup_sgdm_pre_diag(bf16, m, mask) : lookup_sgdm_post_diag(bf16, m, mask);
+        return pre ? lookup_sgdm_pre(bf16, m, mask) : lookup_sgdm_post(bf16, m, mask);
+    }
     return nullptr;
 }
 
 }  // namespace desloc
+
+using desloc::mask_at;
+using desloc::validate_config;
 
 namespace {
 
@@ -56,6 +65,9 @@ struct WorkerRes {
     float *d_norms = nullptr;    // [3][M]: gradient norms, clip factors, relative change
     void **h_snap = nullptr;     // pinned pointer table for desloc_rel_change
     void **d_snap = nullptr;
+    float *d_diag = nullptr;     // diagnostics step: [3][M][nchunks] per-chunk sums of squares
+    double *d_diag_sums = nullptr;  // [3][M][num_tensors]
+    float *d_diag_out = nullptr;    // [3][M][num_tensors] per-tensor norms, then [3][M] totals
 };
 
 void free_worker_res(WorkerRes &r) {
@@ -70,6 +82,9 @@ void free_worker_res(WorkerRes &r) {
     if (r.d_norms) cudaFree(r.d_norms);
     if (r.h_snap) cudaFreeHost(r.h_snap);
     if (r.d_snap) cudaFree(r.d_snap);
+    if (r.d_diag) cudaFree(r.d_diag);
+    if (r.d_diag_sums) cudaFree(r.d_diag_sums);
+    if (r.d_diag_out) cudaFree(r.d_diag_out);
     r = WorkerRes();
 }
 
@@ -92,6 +107,10 @@ cudaError_t make_worker_res(WorkerRes &r, int M, int num_tensors, int64_t nchunk
     if (e == cudaSuccess) e = cudaMemset(r.d_norms, 0, static_cast<size_t>(3) * M * sizeof(float));
     if (e == cudaSuccess) e = cudaMallocHost(&r.h_snap, static_cast<size_t>(nptr) * sizeof(void *));
     if (e == cudaSuccess) e = cudaMalloc(&r.d_snap, static_cast<size_t>(nptr) * sizeof(void *));
+    const size_t ndiag = static_cast<size_t>(desloc::DIAG_KINDS) * M;
+    if (e == cudaSuccess) e = cudaMalloc(&r.d_diag, ndiag * static_cast<size_t>(nchunks) * sizeof(float));
+    if (e == cudaSuccess) e = cudaMalloc(&r.d_diag_sums, ndiag * num_tensors * sizeof(double));
+    if (e == cudaSuccess) e = cudaMalloc(&r.d_diag_out, ndiag * (num_tensors + 1) * sizeof(float));
     for (int i = 0; i < kSlots && e == cudaSuccess; ++i) {
         Slot &s = r.slots[i];
         e = cudaMallocHost(&s.host, static_cast<size_t>(nptr) * sizeof(void *));
@@ -107,7 +126,6 @@ struct desloc_ctx {
     desloc_config cfg{};
     std::vector<int64_t> numel;
     int device = 0;
-    int num_sms = 0;
     int64_t total_elems = 0;
     int64_t nptr = 0;  // M * num_tensors
     desloc::Chunk *d_chunks = nullptr;
@@ -120,7 +138,9 @@ struct desloc_ctx {
     int64_t counters[4] = {0, 0, 0, 0};
     int64_t launches = 0;
     int last_cuda_error = 0;
-    int ctas_per_sm = 0;  // 0: one block per work item; > 0: persistent grid of that many per SM
+    long long *d_tstart = nullptr;  // [num_tensors + 1] first chunk of every tensor
+    bool diag_valid = false;        // a diagnostics step has run since the workers last changed
+    int64_t max_blocks = 0;         // test hook: cap on the grid (0 = one block per work item)
     // desloc_step_host: tensor groups whose copies and kernels are pipelined
     struct Group {
         int32_t k0, k1;   // tensors [k0, k1)
@@ -140,38 +160,6 @@ int cuda_fail(desloc_ctx *ctx, cudaError_t e) {
     return DESLOC_E_CUDA;
 }
 
-bool finite_in(float v, float lo, bool lo_incl, float hi, bool hi_incl) {
-    if (!std::isfinite(v)) return false;
-    if (lo_incl ? v < lo : v <= lo) return false;
-    if (hi_incl ? v > hi : v >= hi) return false;
-    return true;
-}
-
-int validate_config(const desloc_config *c) {
-    if (!c) return DESLOC_E_NULL;
-    if (c->opt != DESLOC_ADAM && c->opt != DESLOC_ADOPT && c->opt != DESLOC_SGDM) return DESLOC_E_INVALID;
-    if (c->grad_dtype != DESLOC_F32 && c->grad_dtype != DESLOC_BF16) return DESLOC_E_INVALID;
-    if (c->flags & ~(DESLOC_FLAG_ADOPT_NORM_CLIP | DESLOC_FLAG_POST_AVERAGE)) return DESLOC_E_INVALID;
-    if ((c->flags & DESLOC_FLAG_ADOPT_NORM_CLIP) && c->opt != DESLOC_ADOPT) return DESLOC_E_INVALID;
-    if (c->M < 1 || c->M > DESLOC_MAX_M) return DESLOC_E_RANGE;
-    if (c->num_tensors < 1) return DESLOC_E_RANGE;
-    if (c->Kx < 0 || c->Ku < 0 || c->Kv < 0) return DESLOC_E_RANGE;
-    if (!finite_in(c->beta1, 0.f, true, 1.f, false)) return DESLOC_E_RANGE;
-    if (c->opt != DESLOC_SGDM && !finite_in(c->beta2, 0.f, true, 1.f, false)) return DESLOC_E_RANGE;
-    if (!finite_in(c->eps, 0.f, true, std::numeric_limits<float>::max(), true)) return DESLOC_E_RANGE;
-    if (!finite_in(c->weight_decay, 0.f, true, std::numeric_limits<float>::max(), true)) return DESLOC_E_RANGE;
-    if (std::isnan(c->clip_rho)) return DESLOC_E_RANGE;
-    return DESLOC_OK;
-}
-
-uint32_t mask_at(const desloc_config *c, int64_t t) {
-    uint32_t m = 0;
-    if (c->Kx > 0 && t % c->Kx == 0) m |= DESLOC_SYNC_X;
-    if (c->Ku > 0 && t % c->Ku == 0) m |= DESLOC_SYNC_U;
-    if (c->opt != DESLOC_SGDM && c->Kv > 0 && t % c->Kv == 0) m |= DESLOC_SYNC_V;
-    return m;
-}
-
 void free_ctx(desloc_ctx *ctx) {
     if (!ctx) return;
     free_worker_res(ctx->res);
@@ -180,6 +168,7 @@ void free_ctx(desloc_ctx *ctx) {
     for (cudaEvent_t ev : ctx->ev_group)
         if (ev) cudaEventDestroy(ev);
     if (ctx->d_chunks) cudaFree(ctx->d_chunks);
+    if (ctx->d_tstart) cudaFree(ctx->d_tstart);
     delete ctx;
 }
 
@@ -210,16 +199,17 @@ int stage_grads(desloc_ctx *ctx, const void *const *grads, cudaStream_t stream, 
 }
 
 // max_norm > 0: norm-based clipping first (two reduction launches), then the step.
+// diag: the step kernel also accumulates the per-chunk sums of squares of g, x_{t+1} and d_t.
 // host_grads != nullptr: the gradients are first copied from host memory into `grads` (device),
 // tensor group by tensor group on the context's copy stream, each group's kernel starting as
 // soon as its copies have landed.
 int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
              const void *const *grads, cudaStream_t stream, float max_norm = 0.f,
-             const void *const *host_grads = nullptr) {
+             const void *const *host_grads = nullptr, bool diag = false) {
     const desloc_config &c = ctx->cfg;
-    if (!std::isfinite(lr_t) || std::isnan(max_norm)) return DESLOC_E_RANGE;
-    const bool nclip = (c.flags & DESLOC_FLAG_ADOPT_NORM_CLIP) != 0;
-    if (nclip && !(clip_bound_t >= 0.f)) return DESLOC_E_RANGE;
+    if (std::isnan(max_norm)) return DESLOC_E_RANGE;
+    int rc = desloc::validate_step(&c, lr_t, clip_bound_t);
+    if (rc != DESLOC_OK) return rc;
     for (int64_t i = 0; i < ctx->nptr; ++i)
         if (!grads[i]) return DESLOC_E_NULL;
 
@@ -230,7 +220,6 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
         e = cudaSetDevice(ctx->device);
         if (e != cudaSuccess) return cuda_fail(ctx, e);
     }
-    int rc = DESLOC_OK;
     do {
         // Under stream capture nothing may be staged through the pinned ring (a replay would
         // read whatever the ring holds by then) and no event of the ring may be recorded.
@@ -274,17 +263,8 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
             d_gscale = ctx->res.d_norms + c.M;
         }
 
-        // The mean of one replica is the replica: M = 1 always runs the local kernel.
-        const uint32_t kmask = (c.M == 1) ? 0u : mask;
-        const bool post = (c.flags & DESLOC_FLAG_POST_AVERAGE) != 0;
-        const bool per_worker_items = (c.M == 1) || (kmask == 0 && c.M > desloc::MAX_MT);
-        const bool generic = kmask != 0 && c.M > desloc::MAX_MT;
-        const void *fn = generic
-                             ? desloc::lookup_generic_kernel(c.opt, post, c.grad_dtype == DESLOC_BF16,
-                                                             static_cast<int>(kmask))
-                             : desloc::lookup_step_kernel(c.opt, post, c.grad_dtype == DESLOC_BF16,
-                                                          c.M, static_cast<int>(kmask));
-        if (!fn) {
+        const desloc::LaunchPlan plan = desloc::plan_launch(c, mask, ctx->nchunks, diag);
+        if (!plan.fn) {
             rc = DESLOC_E_INVALID;
             break;
         }
@@ -298,33 +278,19 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
         if (inline_g)
             for (int64_t i = 0; i < ctx->nptr; ++i) a.g_inline[i] = grads[i];
         a.gscale = d_gscale;
-        a.nt = c.num_tensors;
-        a.M = c.M;
-        a.b1 = c.beta1;
-        a.omb1 = static_cast<float>(1.0 - static_cast<double>(c.beta1));
-        a.b2 = c.beta2;
-        a.omb2 = static_cast<float>(1.0 - static_cast<double>(c.beta2));
-        a.eps = c.eps;
-        a.lam2 = static_cast<float>(static_cast<double>(c.eps) * static_cast<double>(c.eps));
-        a.lr = lr_t;
-        a.lrwd = static_cast<float>(static_cast<double>(lr_t) * static_cast<double>(c.weight_decay));
-        a.rho = c.clip_rho > 0.f ? c.clip_rho : std::numeric_limits<float>::infinity();
-        a.cbound = nclip ? clip_bound_t : std::numeric_limits<float>::infinity();
+        a.diag = diag ? ctx->res.d_diag : nullptr;
+        a.diag_stride = ctx->nchunks;
+        a.diag_chunk0 = 0;
+        desloc::fill_hyper(a, c, lr_t, clip_bound_t);
 
-        const long long nitems =
-            per_worker_items ? ((ctx->nchunks + desloc::LOCAL_SLOTS - 1) / desloc::LOCAL_SLOTS) * c.M
-                             : ctx->nchunks;
-        long long grid = nitems;
-        if (ctx->ctas_per_sm > 0) {
-            const long long cap = static_cast<long long>(ctx->ctas_per_sm) * ctx->num_sms;
-            if (grid > cap) grid = cap;
-        }
-        if (grid > 0x7fffffffLL) grid = 0x7fffffffLL;  // the kernel strides over the rest
-        int kmask_arg = static_cast<int>(kmask);
-        void *params[] = {&a, &kmask_arg};  // the second one is read by the generic kernel only
+        void *params[] = {&a};
+        const auto capped = [ctx](const desloc::LaunchPlan &lp) {
+            const bool cap = lp.strides && ctx->max_blocks > 0 && lp.grid > ctx->max_blocks;
+            return static_cast<unsigned>(cap ? ctx->max_blocks : lp.grid);
+        };
         if (!host_grads) {
-            e = cudaLaunchKernel(fn, dim3(static_cast<unsigned>(grid)), dim3(desloc::BLOCK_THREADS),
-                                 params, 0, stream);
+            e = cudaLaunchKernel(plan.fn, dim3(capped(plan)),
+                                 dim3(desloc::BLOCK_THREADS), params, 0, stream);
             if (e == cudaSuccess) ctx->launches += 1;
         } else {
             // The device gradient buffers may still be read by earlier work on `stream`.
@@ -359,15 +325,9 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
                 if (e != cudaSuccess) break;
                 a.chunks = ctx->d_chunks + grp.c0;
                 a.nchunks = grp.c1 - grp.c0;
-                const long long items =
-                    per_worker_items
-                        ? ((a.nchunks + desloc::LOCAL_SLOTS - 1) / desloc::LOCAL_SLOTS) * c.M
-                        : a.nchunks;
-                long long ggrid = items;
-                if (ctx->ctas_per_sm > 0 && ggrid > static_cast<long long>(ctx->ctas_per_sm) * ctx->num_sms)
-                    ggrid = static_cast<long long>(ctx->ctas_per_sm) * ctx->num_sms;
-                if (ggrid > 0x7fffffffLL) ggrid = 0x7fffffffLL;
-                e = cudaLaunchKernel(fn, dim3(static_cast<unsigned>(ggrid)),
+                a.diag_chunk0 = grp.c0;
+                const desloc::LaunchPlan gp = desloc::plan_launch(c, mask, a.nchunks, diag);
+                e = cudaLaunchKernel(gp.fn, dim3(capped(gp)),
                                      dim3(desloc::BLOCK_THREADS), params, 0, stream);
                 if (e == cudaSuccess) ctx->launches += 1;
             }
@@ -385,6 +345,7 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
             }
             s.in_flight = true;
         }
+        if (diag) ctx->diag_valid = true;
         ctx->counters[0] += 1;
         ctx->counters[1] += (mask & DESLOC_SYNC_X) ? 1 : 0;
         ctx->counters[2] += (mask & DESLOC_SYNC_U) ? 1 : 0;
@@ -436,37 +397,31 @@ int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *const *x, f
     if (cuda_device < 0) return DESLOC_E_RANGE;
     const int64_t nptr = static_cast<int64_t>(cfg->M) * cfg->num_tensors;
     int64_t total = 0;
-    for (int32_t k = 0; k < cfg->num_tensors; ++k) {
-        if (cfg->numel[k] < 1) return DESLOC_E_RANGE;
-        if (cfg->numel[k] > (INT64_MAX >> 4) - total) return DESLOC_E_RANGE;
-        total += cfg->numel[k];
-    }
+    rc = desloc::validate_numel(cfg, &total);
+    if (rc != DESLOC_OK) return rc;
     for (int64_t i = 0; i < nptr; ++i) {
         if (!x[i] || !u[i]) return DESLOC_E_NULL;
         if (cfg->opt != DESLOC_SGDM && !v[i]) return DESLOC_E_NULL;
     }
+    const int64_t chunk_elems = desloc::chunk_elems_for(cfg->numel, cfg->num_tensors);
+    const int64_t nchunks = desloc::count_chunks(cfg->numel, cfg->num_tensors, chunk_elems);
+    // one thread block per chunk (or per worker and group of chunks): the grid must fit
+    if (nchunks > 0x7fffffffLL ||
+        (nchunks / desloc::LOCAL_SLOTS + 1) * static_cast<int64_t>(cfg->M) > 0x7fffffffLL)
+        return DESLOC_E_RANGE;
 
     desloc_ctx *ctx = new (std::nothrow) desloc_ctx();
     if (!ctx) return DESLOC_E_NOMEM;
     std::vector<desloc::Chunk> chunks;
-    // Small problems (fewer full-size chunks than two per SM of a B200) are latency-bound:
-    // quarter-size chunks spread them over four times as many blocks, one tile per thread.
-    int64_t full_chunks = 0;
-    for (int32_t k = 0; k < cfg->num_tensors; ++k)
-        full_chunks += (cfg->numel[k] + desloc::CHUNK_ELEMS - 1) / desloc::CHUNK_ELEMS;
-    const int64_t chunk_elems = full_chunks < 2 * 148 ? desloc::CHUNK_ELEMS / 4 : desloc::CHUNK_ELEMS;
+    std::vector<long long> tstart;
     try {
         ctx->numel.assign(cfg->numel, cfg->numel + cfg->num_tensors);
         ctx->last_grads.assign(static_cast<size_t>(nptr), nullptr);
+        chunks.resize(static_cast<size_t>(nchunks));
+        desloc::fill_chunks(cfg->numel, cfg->num_tensors, chunk_elems, chunks.data());
+        tstart.assign(static_cast<size_t>(cfg->num_tensors) + 1, 0);
         for (int32_t k = 0; k < cfg->num_tensors; ++k)
-            for (int64_t s = 0; s < cfg->numel[k]; s += chunk_elems) {
-                desloc::Chunk ch;
-                ch.tensor = k;
-                ch.start = s;
-                const int64_t left = cfg->numel[k] - s;
-                ch.count = static_cast<int32_t>(left < chunk_elems ? left : chunk_elems);
-                chunks.push_back(ch);
-            }
+            tstart[k + 1] = tstart[k] + (cfg->numel[k] + chunk_elems - 1) / chunk_elems;
     } catch (const std::bad_alloc &) {
         delete ctx;
         return DESLOC_E_NOMEM;
@@ -476,16 +431,18 @@ int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *const *x, f
     ctx->device = cuda_device;
     ctx->total_elems = total;
     ctx->nptr = nptr;
-    ctx->nchunks = static_cast<int64_t>(chunks.size());
+    ctx->nchunks = nchunks;
 
     int dev_before = -1;
     cudaError_t e = cudaGetDevice(&dev_before);
     if (e == cudaSuccess && dev_before != cuda_device) e = cudaSetDevice(cuda_device);
-    if (e == cudaSuccess)
-        e = cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, cuda_device);
     if (e == cudaSuccess) e = cudaMalloc(&ctx->d_chunks, chunks.size() * sizeof(desloc::Chunk));
     if (e == cudaSuccess)
         e = cudaMemcpy(ctx->d_chunks, chunks.data(), chunks.size() * sizeof(desloc::Chunk),
+                       cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_tstart, tstart.size() * sizeof(long long));
+    if (e == cudaSuccess)
+        e = cudaMemcpy(ctx->d_tstart, tstart.data(), tstart.size() * sizeof(long long),
                        cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_entry, cudaEventDisableTiming);
@@ -527,6 +484,7 @@ int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *const *x, f
 
 int desloc_step(desloc_ctx *ctx, int64_t t, float lr_t, float clip_bound_t,
                 const void *const *grads, void *stream, uint32_t *mask_out) {
+    desloc::NvtxRange range("desloc_step");
     if (!ctx || !grads) return DESLOC_E_NULL;
     if (t < 0) return DESLOC_E_RANGE;
     const uint32_t mask = mask_at(&ctx->cfg, t);
@@ -535,9 +493,48 @@ int desloc_step(desloc_ctx *ctx, int64_t t, float lr_t, float clip_bound_t,
     return rc;
 }
 
+int desloc_step_diag(desloc_ctx *ctx, int64_t t, float lr_t, float clip_bound_t, float max_norm,
+                     const void *const *grads, void *stream, uint32_t *mask_out) {
+    desloc::NvtxRange range("desloc_step_diag");
+    if (!ctx || !grads) return DESLOC_E_NULL;
+    if (t < 0 || !(max_norm >= 0.f) || !std::isfinite(max_norm)) return DESLOC_E_RANGE;
+    const uint32_t mask = mask_at(&ctx->cfg, t);
+    const int rc = run_step(ctx, mask, lr_t, clip_bound_t, grads, static_cast<cudaStream_t>(stream),
+                            max_norm, nullptr, true);
+    if (rc == DESLOC_OK && mask_out) *mask_out = mask;
+    return rc;
+}
+
+int desloc_get_diag_norms(desloc_ctx *ctx, float *per_tensor_out, float *total_out, void *stream) {
+    if (!ctx) return DESLOC_E_NULL;
+    if (!ctx->diag_valid) return DESLOC_E_INVALID;
+    const desloc_config &c = ctx->cfg;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int dev_before = -1;
+    cudaError_t e = cudaGetDevice(&dev_before);
+    if (e == cudaSuccess && dev_before != ctx->device) e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    const size_t rows = static_cast<size_t>(desloc::DIAG_KINDS) * c.M;
+    float *d_per = ctx->res.d_diag_out, *d_tot = ctx->res.d_diag_out + rows * c.num_tensors;
+    e = desloc::launch_diag_norms(ctx->res.d_diag, ctx->nchunks, ctx->d_tstart, c.num_tensors, c.M,
+                                  ctx->res.d_diag_sums, d_per, d_tot, st);
+    if (e == cudaSuccess) {
+        ctx->launches += 2;
+        if (per_tensor_out)
+            e = cudaMemcpyAsync(per_tensor_out, d_per, rows * c.num_tensors * sizeof(float),
+                                cudaMemcpyDeviceToHost, st);
+    }
+    if (e == cudaSuccess && total_out)
+        e = cudaMemcpyAsync(total_out, d_tot, rows * sizeof(float), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (dev_before != ctx->device) cudaSetDevice(dev_before);
+    return e == cudaSuccess ? DESLOC_OK : cuda_fail(ctx, e);
+}
+
 int desloc_step_host(desloc_ctx *ctx, int64_t t, float lr_t, float clip_bound_t,
                      const void *const *host_grads, void *const *dev_grads, void *stream,
                      uint32_t *mask_out) {
+    desloc::NvtxRange range("desloc_step_host");
     if (!ctx || !host_grads || !dev_grads) return DESLOC_E_NULL;
     if (t < 0) return DESLOC_E_RANGE;
     for (int64_t i = 0; i < ctx->nptr; ++i)
@@ -552,6 +549,7 @@ int desloc_step_host(desloc_ctx *ctx, int64_t t, float lr_t, float clip_bound_t,
 
 int desloc_step_masked(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
                        const void *const *grads, void *stream) {
+    desloc::NvtxRange range("desloc_step_masked");
     if (!ctx || !grads) return DESLOC_E_NULL;
     if (mask & ~7u) return DESLOC_E_INVALID;
     if (ctx->cfg.opt == DESLOC_SGDM && (mask & DESLOC_SYNC_V)) return DESLOC_E_INVALID;
@@ -561,6 +559,7 @@ int desloc_step_masked(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bo
 int desloc_step_normclip(desloc_ctx *ctx, int64_t t, float lr_t, float clip_bound_t,
                          float max_norm, const void *const *grads, void *stream,
                          uint32_t *mask_out) {
+    desloc::NvtxRange range("desloc_step_normclip");
     if (!ctx || !grads) return DESLOC_E_NULL;
     if (t < 0 || !(max_norm > 0.f) || !std::isfinite(max_norm)) return DESLOC_E_RANGE;
     const uint32_t mask = mask_at(&ctx->cfg, t);
@@ -669,6 +668,7 @@ int desloc_set_workers(desloc_ctx *ctx, int32_t M_new, int32_t first_new, float 
         ctx->nptr = nptr_new;
         ctx->next_slot = 0;
         ctx->cur_slot = -1;
+        ctx->diag_valid = false;
     } else {
         free_worker_res(fresh);
         rc = (e == cudaErrorMemoryAllocation) ? DESLOC_E_NOMEM : cuda_fail(ctx, e);
@@ -698,10 +698,10 @@ int desloc_get_counters(const desloc_ctx *ctx, int64_t out[4]) {
 
 int64_t desloc_get_launch_count(const desloc_ctx *ctx) { return ctx ? ctx->launches : 0; }
 
-int desloc_set_launch_shape(desloc_ctx *ctx, int32_t ctas_per_sm) {
+int desloc_testing_set_max_blocks(desloc_ctx *ctx, int64_t max_blocks) {
     if (!ctx) return DESLOC_E_NULL;
-    if (ctas_per_sm < 0 || ctas_per_sm > 32) return DESLOC_E_RANGE;
-    ctx->ctas_per_sm = ctas_per_sm;
+    if (max_blocks < 0) return DESLOC_E_RANGE;
+    ctx->max_blocks = max_blocks;
     return DESLOC_OK;
 }
 

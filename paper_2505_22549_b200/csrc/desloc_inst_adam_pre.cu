@@ -3,7 +3,6 @@
 
 namespace desloc {
 const void *lookup_adam_pre(bool bf16, int mt, int mask) {
-    if (mt == 1) return mask == 0 ? lookup_local<OPT_ADAM>(bf16) : nullptr;
-    return lookup_sync<OPT_ADAM, false>(bf16, mt, mask);
+    return lookup_unit<OPT_ADAM, false, false>(bf16, mt, mask);
 }
 }  // namespace desloc

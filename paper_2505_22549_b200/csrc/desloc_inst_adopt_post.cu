@@ -3,7 +3,6 @@
 
 namespace desloc {
 const void *lookup_adopt_post(bool bf16, int mt, int mask) {
-
-    return lookup_sync<OPT_ADOPT, true>(bf16, mt, mask);
+    return lookup_unit<OPT_ADOPT, true, false>(bf16, mt, mask);
 }
 }  // namespace desloc

@@ -1,0 +1,8 @@
+// desloc_step_kernel instantiations: ADOPT, post-average ordering, with norm diagnostics.
+#include "desloc_inst.cuh"
+
+namespace desloc {
+const void *lookup_adopt_post_diag(bool bf16, int mt, int mask) {
+    return lookup_unit<OPT_ADOPT, true, true>(bf16, mt, mask);
+}
+}  // namespace desloc

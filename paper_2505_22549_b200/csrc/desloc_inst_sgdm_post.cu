@@ -3,7 +3,6 @@
 
 namespace desloc {
 const void *lookup_sgdm_post(bool bf16, int mt, int mask) {
-
-    return lookup_sync<OPT_SGDM, true>(bf16, mt, mask);
+    return lookup_unit<OPT_SGDM, true, false>(bf16, mt, mask);
 }
 }  // namespace desloc

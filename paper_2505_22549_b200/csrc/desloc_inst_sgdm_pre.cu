@@ -3,7 +3,6 @@
 
 namespace desloc {
 const void *lookup_sgdm_pre(bool bf16, int mt, int mask) {
-    if (mt == 1) return mask == 0 ? lookup_local<OPT_SGDM>(bf16) : nullptr;
-    return lookup_sync<OPT_SGDM, false>(bf16, mt, mask);
+    return lookup_unit<OPT_SGDM, false, false>(bf16, mt, mask);
 }
 }  // namespace desloc

@@ -1,0 +1,145 @@
+// Host-side pieces shared by the context path (desloc_host.cu) and the allocation-free entry
+// point (desloc_static.cu): argument validation, the sync schedule, the chunk-size rule and the
+// kernel-argument block, so that both paths validate, plan and launch identically.
+#pragma once
+#include <cmath>
+#include <cstdint>
+#include <limits>
+
+#include <nvtx3/nvToolsExt.h>
+
+#include "../../include/desloc.h"
+#include "desloc_kernels.cuh"
+
+namespace desloc {
+
+// A named range around every step call, visible to tools that record NVTX (no cost otherwise).
+struct NvtxRange {
+    explicit NvtxRange(const char *name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+    NvtxRange(const NvtxRange &) = delete;
+    NvtxRange &operator=(const NvtxRange &) = delete;
+};
+
+inline bool finite_in(float v, float lo, bool lo_incl, float hi, bool hi_incl) {
+    if (!std::isfinite(v)) return false;
+    if (lo_incl ? v < lo : v <= lo) return false;
+    if (hi_incl ? v > hi : v >= hi) return false;
+    return true;
+}
+
+// Everything about a desloc_config that can be checked without looking at numel or the device.
+inline int validate_config(const desloc_config *c) {
+    if (!c) return DESLOC_E_NULL;
+    if (c->opt != DESLOC_ADAM && c->opt != DESLOC_ADOPT && c->opt != DESLOC_SGDM) return DESLOC_E_INVALID;
+    if (c->grad_dtype != DESLOC_F32 && c->grad_dtype != DESLOC_BF16) return DESLOC_E_INVALID;
+    if (c->flags & ~(DESLOC_FLAG_ADOPT_NORM_CLIP | DESLOC_FLAG_POST_AVERAGE)) return DESLOC_E_INVALID;
+    if ((c->flags & DESLOC_FLAG_ADOPT_NORM_CLIP) && c->opt != DESLOC_ADOPT) return DESLOC_E_INVALID;
+    if (c->M < 1 || c->M > DESLOC_MAX_M) return DESLOC_E_RANGE;
+    if (c->num_tensors < 1) return DESLOC_E_RANGE;
+    if (c->Kx < 0 || c->Ku < 0 || c->Kv < 0) return DESLOC_E_RANGE;
+    if (!finite_in(c->beta1, 0.f, true, 1.f, false)) return DESLOC_E_RANGE;
+    if (c->opt != DESLOC_SGDM && !finite_in(c->beta2, 0.f, true, 1.f, false)) return DESLOC_E_RANGE;
+    if (!finite_in(c->eps, 0.f, true, std::numeric_limits<float>::max(), true)) return DESLOC_E_RANGE;
+    if (!finite_in(c->weight_decay, 0.f, true, std::numeric_limits<float>::max(), true)) return DESLOC_E_RANGE;
+    if (std::isnan(c->clip_rho)) return DESLOC_E_RANGE;
+    return DESLOC_OK;
+}
+
+// numel[k] >= 1 for every tensor and a total that cannot overflow the byte arithmetic.
+inline int validate_numel(const desloc_config *c, int64_t *total_out) {
+    if (!c->numel) return DESLOC_E_NULL;
+    int64_t total = 0;
+    for (int32_t k = 0; k < c->num_tensors; ++k) {
+        if (c->numel[k] < 1) return DESLOC_E_RANGE;
+        if (c->numel[k] > (INT64_MAX >> 4) - total) return DESLOC_E_RANGE;
+        total += c->numel[k];
+    }
+    if (total_out) *total_out = total;
+    return DESLOC_OK;
+}
+
+// Per-step scalar arguments.
+inline int validate_step(const desloc_config *c, float lr_t, float clip_bound_t) {
+    if (!std::isfinite(lr_t)) return DESLOC_E_RANGE;
+    if ((c->flags & DESLOC_FLAG_ADOPT_NORM_CLIP) && !(clip_bound_t >= 0.f)) return DESLOC_E_RANGE;
+    return DESLOC_OK;
+}
+
+// Algorithm 1's three "t mod K = 0" tests, t from 0; K = 0 never syncs; SGDM has no second state.
+inline uint32_t mask_at(const desloc_config *c, int64_t t) {
+    uint32_t m = 0;
+    if (c->Kx > 0 && t % c->Kx == 0) m |= DESLOC_SYNC_X;
+    if (c->Ku > 0 && t % c->Ku == 0) m |= DESLOC_SYNC_U;
+    if (c->opt != DESLOC_SGDM && c->Kv > 0 && t % c->Kv == 0) m |= DESLOC_SYNC_V;
+    return m;
+}
+
+// Chunk length for a tensor list.  Small problems (fewer full-size chunks than two per SM of a
+// B200) are latency-bound: quarter-size chunks spread them over four times as many blocks.
+inline int64_t chunk_elems_for(const int64_t *numel, int32_t num_tensors) {
+    int64_t full = 0;
+    for (int32_t k = 0; k < num_tensors; ++k) full += (numel[k] + CHUNK_ELEMS - 1) / CHUNK_ELEMS;
+    return full < 2 * 148 ? CHUNK_ELEMS / 4 : CHUNK_ELEMS;
+}
+
+inline int64_t count_chunks(const int64_t *numel, int32_t num_tensors, int64_t chunk_elems) {
+    int64_t n = 0;
+    for (int32_t k = 0; k < num_tensors; ++k) n += (numel[k] + chunk_elems - 1) / chunk_elems;
+    return n;
+}
+
+// Writes the chunk table for the list (every tensor starts a new chunk); `out` has room for
+// count_chunks() entries.
+inline void fill_chunks(const int64_t *numel, int32_t num_tensors, int64_t chunk_elems, Chunk *out) {
+    int64_t c = 0;
+    for (int32_t k = 0; k < num_tensors; ++k)
+        for (int64_t s = 0; s < numel[k]; s += chunk_elems) {
+            const int64_t left = numel[k] - s;
+            out[c].tensor = k;
+            out[c].count = static_cast<int32_t>(left < chunk_elems ? left : chunk_elems);
+            out[c].start = s;
+            ++c;
+        }
+}
+
+// The hyper-parameter part of the kernel arguments (tables and sizes are the caller's).
+inline void fill_hyper(StepArgs &a, const desloc_config &c, float lr_t, float clip_bound_t) {
+    a.nt = c.num_tensors;
+    a.M = c.M;
+    a.b1 = c.beta1;
+    a.omb1 = static_cast<float>(1.0 - static_cast<double>(c.beta1));
+    a.b2 = c.beta2;
+    a.omb2 = static_cast<float>(1.0 - static_cast<double>(c.beta2));
+    a.eps = c.eps;
+    a.lam2 = static_cast<float>(static_cast<double>(c.eps) * static_cast<double>(c.eps));
+    a.lr = lr_t;
+    a.lrwd = static_cast<float>(static_cast<double>(lr_t) * static_cast<double>(c.weight_decay));
+    a.rho = c.clip_rho > 0.f ? c.clip_rho : std::numeric_limits<float>::infinity();
+    a.cbound = (c.flags & DESLOC_FLAG_ADOPT_NORM_CLIP) ? clip_bound_t
+                                                       : std::numeric_limits<float>::infinity();
+}
+
+// Which kernel a step of this configuration runs, and over how many blocks.
+struct LaunchPlan {
+    const void *fn = nullptr;
+    long long grid = 0;
+    bool strides = true;  // a smaller grid may stride over the work items (not the runtime-M kernel)
+};
+
+inline LaunchPlan plan_launch(const desloc_config &c, uint32_t mask, long long nchunks, bool diag) {
+    LaunchPlan p;
+    // The mean of one replica is the replica: M = 1 always runs the local kernel.
+    const uint32_t kmask = (c.M == 1) ? 0u : mask;
+    const bool post = (c.flags & DESLOC_FLAG_POST_AVERAGE) != 0;
+    const bool bf16 = c.grad_dtype == DESLOC_BF16;
+    const bool per_worker_items = (c.M == 1) || (kmask == 0 && c.M > MAX_MT);
+    const bool generic = kmask != 0 && c.M > MAX_MT;
+    p.fn = generic ? lookup_generic_kernel(c.opt, post, bf16, static_cast<int>(kmask), diag)
+                   : lookup_step_kernel(c.opt, post, bf16, c.M, static_cast<int>(kmask), diag);
+    p.strides = !generic;
+    p.grid = per_worker_items ? ((nchunks + LOCAL_SLOTS - 1) / LOCAL_SLOTS) * c.M : nchunks;
+    return p;
+}
+
+}  // namespace desloc

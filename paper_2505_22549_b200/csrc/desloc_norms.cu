@@ -1,6 +1,7 @@
 // Reductions around the DES-LOC step: per-worker gradient norms for norm-based clipping (the
-// clipping the paper's language-model runs used) and the relative rate of change of a state,
-// ||s_now - s_then||_2 / ||s_then||_2 (Section 5.1, "Metrics").
+// clipping the paper's language-model runs used), the relative rate of change of a state,
+// ||s_now - s_then||_2 / ||s_then||_2 (Section 5.1, "Metrics"), and the finalisation of the
+// per-tensor gradient / parameter / update norms a diagnostics step accumulated.
 //
 // Both are two-stage and deterministic: stage 1 writes one fp32 partial per (worker, chunk)
 // -- per-thread sums of up to 16 squares, a shuffle tree, then the eight warp sums in order;
@@ -120,7 +121,7 @@ sumsq_kernel(const Chunk *chunks, long long nchunks, const void *const *g, int n
                     if (wide[k + j]) {
 #pragma unroll
                         for (int l = 0; l < LPC; ++l)
-                            r[j][l] = ld_stream(wide[k + j] + tid + l * BLOCK_THREADS);
+                            r[j][l] = *(wide[k + j] + tid + l * BLOCK_THREADS);
                     }
                 }
 #pragma unroll
@@ -201,7 +202,8 @@ relchange_kernel(const Chunk *chunks, long long nchunks, const float *const *now
 
 // One block per row: out_sum[row] = sum of partial[row * n .. +n) in fp64, fixed pattern
 // (thread i adds entries i, i+256, ... in order; then a shared-memory tree).
-__device__ __forceinline__ double row_sum_f64(const float *row, long long n, double *sh) {
+template <typename T>
+__device__ __forceinline__ double row_sum_f64(const T *row, long long n, double *sh) {
     double acc = 0.0;
     for (long long i = threadIdx.x; i < n; i += BLOCK_THREADS) acc += static_cast<double>(row[i]);
     sh[threadIdx.x] = acc;
@@ -258,6 +260,31 @@ mean_fill_kernel(const Chunk *chunks, long long nchunks, const float *const *src
     }
 }
 
+// Norm diagnostics of a DIAG step.  partial[(kind * M + m) * stride + c] holds the sum of
+// squares of chunk c; tstart[k] .. tstart[k + 1] are the chunks of tensor k.  One block per
+// (tensor, worker, kind): fp64 sum of the tensor's chunks, its root as the per-tensor norm.
+__global__ void __launch_bounds__(BLOCK_THREADS)
+diag_tensor_kernel(const float *partial, long long stride, const long long *tstart, int nt, int M,
+                   double *sums, float *norms) {
+    __shared__ double sh[BLOCK_THREADS];
+    const int k = blockIdx.x, m = blockIdx.y, kind = blockIdx.z;
+    const long long row = static_cast<long long>(kind) * M + m;
+    const double ss = row_sum_f64(partial + row * stride + tstart[k], tstart[k + 1] - tstart[k], sh);
+    if (threadIdx.x == 0) {
+        sums[row * nt + k] = ss;
+        norms[row * nt + k] = static_cast<float>(sqrt(ss));
+    }
+}
+
+// One block per (kind, worker): the whole-model norm from the per-tensor sums of squares.
+__global__ void __launch_bounds__(BLOCK_THREADS)
+diag_total_kernel(const double *sums, int nt, float *totals) {
+    __shared__ double sh[BLOCK_THREADS];
+    const long long row = blockIdx.x;
+    const double ss = row_sum_f64(sums + row * nt, nt, sh);
+    if (threadIdx.x == 0) totals[row] = static_cast<float>(sqrt(ss));
+}
+
 unsigned grid_for(long long nitems) {
     return static_cast<unsigned>(nitems < 0x7fffffffLL ? (nitems > 0 ? nitems : 1) : 0x7fffffffLL);
 }
@@ -287,6 +314,17 @@ cudaError_t launch_rel_change(const Chunk *chunks, long long nchunks, const floa
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     relchange_finalize_kernel<<<M, BLOCK_THREADS, 0, stream>>>(partial, nchunks, M, out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_diag_norms(const float *partial, long long stride, const long long *tstart,
+                              int nt, int M, double *sums, float *per_tensor, float *totals,
+                              cudaStream_t stream) {
+    diag_tensor_kernel<<<dim3(nt, M, DIAG_KINDS), BLOCK_THREADS, 0, stream>>>(partial, stride, tstart,
+                                                                            nt, M, sums, per_tensor);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    diag_total_kernel<<<DIAG_KINDS * M, BLOCK_THREADS, 0, stream>>>(sums, nt, totals);
     return cudaGetLastError();
 }
 

@@ -15,6 +15,13 @@ cudaError_t launch_rel_change(const Chunk *chunks, long long nchunks, const floa
                               const float *const *then, int nt, int M, float *partial, float *out,
                               cudaStream_t stream);
 
+// Norms of a diagnostics step: partial [DIAG_KINDS][M][stride] per-chunk sums of squares,
+// tstart [nt + 1] first chunk of every tensor; writes sums [DIAG_KINDS][M][nt] (fp64 scratch),
+// per_tensor [DIAG_KINDS][M][nt] and totals [DIAG_KINDS][M] (floats), all on the device.
+cudaError_t launch_diag_norms(const float *partial, long long stride, const long long *tstart,
+                              int nt, int M, double *sums, float *per_tensor, float *totals,
+                              cudaStream_t stream);
+
 // Every element of the m_dst destination replicas := mean over the m_src source replicas.
 // src / dst are device tables indexed [m * nt + tensor].
 cudaError_t launch_mean_fill(const Chunk *chunks, long long nchunks, const float *const *src,

@@ -8,6 +8,13 @@ import torch
 from . import binding as B
 
 
+class BoundGrads:
+    """Gradient tensors already checked and marshalled (see DesLoc.bind_grads)."""
+
+    def __init__(self, array, keep):
+        self.array, self._keep = array, keep
+
+
 class DesLoc:
     """M worker replicas of a tensor list, stepped by the CUDA library.
 
@@ -44,7 +51,15 @@ class DesLoc:
         self._gkey = None
         self._garr = None
 
-    def _grad_array(self, grads: Sequence[Sequence[torch.Tensor]]):
+    def bind_grads(self, grads: Sequence[Sequence[torch.Tensor]]):
+        """Check a set of gradient tensors once and return a handle every step method accepts in
+        place of the nested lists: a loop that reuses its gradient buffers then pays no
+        per-step marshalling.  The handle keeps the tensors alive."""
+        return BoundGrads(self._grad_array(grads), grads)
+
+    def _grad_array(self, grads):
+        if isinstance(grads, BoundGrads):
+            return grads.array
         want = torch.bfloat16 if self.grad_dtype == B.DESLOC_BF16 else torch.float32
         ptrs: List[int] = []
         for lst in grads:
@@ -69,6 +84,19 @@ class DesLoc:
         stream = torch.cuda.current_stream(self.device).cuda_stream
         return B.desloc_step_normclip(self.ctx, t, lr, clip_bound, max_norm,
                                       self._grad_array(grads), stream)
+
+    def step_diag(self, t: int, lr: float, grads, max_norm: float = 0.0, clip_bound: float = 0.0) -> int:
+        """Step t that also accumulates the gradient, parameter and update norms (read them with
+        diag_norms()); max_norm > 0 adds norm-based clipping in front."""
+        stream = torch.cuda.current_stream(self.device).cuda_stream
+        return B.desloc_step_diag(self.ctx, t, lr, clip_bound, max_norm, self._grad_array(grads),
+                                  stream)
+
+    def diag_norms(self):
+        """(per_tensor [3][M][num_tensors], total [3][M]) of the latest step_diag; kind 0 =
+        gradient as read, 1 = new parameters, 2 = update d_t.  Synchronises the current stream."""
+        stream = torch.cuda.current_stream(self.device).cuda_stream
+        return B.desloc_get_diag_norms(self.ctx, self.M, len(self.numel), stream)
 
     def grad_norms(self):
         """(norms, clip factors) of the latest step_normclip; synchronises the current stream."""
@@ -123,9 +151,6 @@ class DesLoc:
 
     def launches(self) -> int:
         return B.desloc_get_launch_count(self.ctx)
-
-    def set_launch_shape(self, ctas_per_sm: int) -> None:
-        B.desloc_set_launch_shape(self.ctx, ctas_per_sm)
 
     def close(self) -> None:
         if self.ctx is not None:

@@ -21,12 +21,17 @@ def d():
 
 
 def test_library_exports_every_declared_symbol(d):
-    header = open(os.path.join(ROOT, "include", "desloc.h")).read()
-    names = re.findall(r"DESLOC_API\s+[\w\s\*]+?\b(desloc_\w+)\s*\(", header)
-    assert len(names) >= 12 and len(set(names)) == len(names)
+    names = []
+    for h in ("desloc.h", "desloc_testing.h"):
+        header = open(os.path.join(ROOT, "include", h)).read()
+        names += re.findall(r"DESLOC_API\s+[\w\s\*]+?\b(desloc_\w+)\s*\(", header)
+    assert len(names) >= 19 and len(set(names)) == len(names)
+    for must in ("desloc_create", "desloc_step", "desloc_destroy", "desloc_step_diag",
+                 "desloc_get_diag_norms", "desloc_step_static", "desloc_testing_set_max_blocks"):
+        assert must in names
     L = d.raw_lib()
     for n in names:
-        assert hasattr(L, n), f"{n} declared in desloc.h but not exported"
+        assert hasattr(L, n), f"{n} declared in a header but not exported"
 
 
 def test_header_is_plain_c_and_a_c_program_links(d, tmp_path):
@@ -141,3 +146,56 @@ def test_no_cpu_fallback_without_a_device(d):
     with pytest.raises(d.DeslocError) as e:
         d.desloc_create(cfg, [16], [16], [16], 0)
     assert e.value.status in (d.DESLOC_E_CUDA, d.DESLOC_E_NOMEM)
+
+
+def test_diag_entry_points_reject_bad_arguments_without_a_device(d):
+    L = d.raw_lib()
+    assert L.desloc_step_diag(None, 0, 0.1, 0.0, 0.0, None, None, None) == d.DESLOC_E_NULL
+    assert L.desloc_get_diag_norms(None, None, None, None) == d.DESLOC_E_NULL
+    assert L.desloc_testing_set_max_blocks(None, 0) == d.DESLOC_E_NULL
+
+
+STATIC_BAD = [
+    (dict(M=0), "DESLOC_E_RANGE"), (dict(M=9), "DESLOC_E_TOO_LARGE"), (dict(M=257), "DESLOC_E_RANGE"),
+    (dict(beta1=1.0), "DESLOC_E_RANGE"), (dict(beta2=float("nan")), "DESLOC_E_RANGE"),
+    (dict(eps=-1.0), "DESLOC_E_RANGE"), (dict(Kv=-2), "DESLOC_E_RANGE"),
+    (dict(opt=7), "DESLOC_E_INVALID"), (dict(grad_dtype=5), "DESLOC_E_INVALID"),
+    (dict(flags=8), "DESLOC_E_INVALID"), (dict(flags=1), "DESLOC_E_INVALID"),
+    (dict(numel=[4, 0]), "DESLOC_E_RANGE"),
+    (dict(numel=[1] * 1025), "DESLOC_E_TOO_LARGE"),                 # 2 x 1025 pointers
+    (dict(M=1, numel=[16384 * 4096 + 1]), "DESLOC_E_TOO_LARGE"),    # one chunk too many
+]
+
+
+@pytest.mark.parametrize("kw,status", STATIC_BAD)
+def test_static_entry_point_rejects_bad_arguments_before_any_cuda_call(d, kw, status):
+    """desloc_step_static() validates everything first: these calls must return their status on
+    a machine with no GPU at all (nothing may reach the CUDA runtime)."""
+    args = dict(M=2, numel=[4, 4], opt="adam", grad_dtype="f32")
+    args.update(kw)
+    cfg = d.make_config(**args)
+    n = max(1, cfg.M) * len(args["numel"])
+    with pytest.raises(d.DeslocError) as e:
+        d.desloc_step_static(cfg, [16] * n, [16] * n, [16] * n, [16] * n, 0, 1e-3, 0.0, 0)
+    assert e.value.status == getattr(d, status)
+
+
+def test_static_entry_point_rejects_nulls_and_bad_step_arguments(d):
+    cfg = d.make_config(2, [4], "adam", "f32")
+    ok = [16, 16]
+    for x, u, v, g in [(None, ok, ok, ok), (ok, None, ok, ok), (ok, ok, None, ok), (ok, ok, ok, None),
+                       ([16, 0], ok, ok, ok), (ok, ok, [0, 16], ok), (ok, ok, ok, [16, 0])]:
+        with pytest.raises(d.DeslocError) as e:
+            d.desloc_step_static(cfg, x, u, v, g, 0, 1e-3, 0.0, 0)
+        assert e.value.status == d.DESLOC_E_NULL
+    for t, lr, dev in [(-1, 1e-3, 0), (0, float("inf"), 0), (0, 1e-3, -1), (0, 1e-3, 64)]:
+        with pytest.raises(d.DeslocError) as e:
+            d.desloc_step_static(cfg, ok, ok, ok, ok, t, lr, 0.0, dev)
+        assert e.value.status == d.DESLOC_E_RANGE
+    assert d.raw_lib().desloc_step_static(None, None, None, None, None, 0, 0.1, 0.0, 0, None, None) \
+        == d.DESLOC_E_NULL
+    # the ADOPT bound must be a number >= 0 when its flag is set
+    cfg = d.make_config(2, [4], "adopt", "f32", flags=d.DESLOC_FLAG_ADOPT_NORM_CLIP)
+    with pytest.raises(d.DeslocError) as e:
+        d.desloc_step_static(cfg, ok, ok, ok, ok, 0, 1e-3, float("nan"), 0)
+    assert e.value.status == d.DESLOC_E_RANGE

@@ -110,3 +110,32 @@ def test_shard_tensor_list_properties():
                 assert (max(sizes) - min(sizes)) / max(sizes) < 1e-3
     with pytest.raises(ValueError):
         dd.shard_tensor_list([4], 2, 2)
+
+
+def test_bench_gpus_n_starts_n_ranks(monkeypatch):
+    """`python bench.py --gpus N` outside torchrun must become N ranks (one per GPU) through
+    torch.distributed.run on 127.0.0.1; under torchrun (WORLD_SIZE set) it must not re-launch."""
+    import importlib
+    import os
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    sys.path.insert(0, root)
+    bench = importlib.import_module("bench")
+    cmd = bench.launcher_command(4, ["--gpus", "4", "--steps", "5", "--warmup", "3"], port=29555)
+    assert cmd[:3] == [sys.executable, "-m", "torch.distributed.run"]
+    assert "--nnodes=1" in cmd and "--nproc-per-node=4" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[cmd.index("--master-port") + 1] == "29555"
+    assert cmd[-7] == os.path.join(root, "bench.py") and cmd[-6:] == ["--gpus", "4", "--steps", "5", "--warmup", "3"]
+    assert bench.launcher_command(2, [])[-1].endswith("bench.py")          # picks a free port itself
+
+    calls = []
+    monkeypatch.setattr(bench.subprocess, "call", lambda c: calls.append(c) or 0)
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    assert bench.main(["--gpus", "2", "--steps", "3"]) == 0
+    assert len(calls) == 1 and "--nproc-per-node=2" in calls[0] and calls[0][-4:] == ["--gpus", "2", "--steps", "3"]
+    # as a rank of a torchrun job: no second launch (the reference arm returns at once off rank 0)
+    monkeypatch.setenv("WORLD_SIZE", "2")
+    monkeypatch.setenv("RANK", "1")
+    assert bench.main(["--gpus", "2", "--impl", "reference", "--steps", "1"]) == 0
+    assert len(calls) == 1

@@ -34,14 +34,14 @@ def make_engine(d, w, st, post=False):
 
 
 def run_both(w, T, align=4, byte_shift=0, post=False, v_init=0.0, identical=False,
-             forced_masks=None, lr_of_t=None, ctas_per_sm=0):
+             forced_masks=None, lr_of_t=None, max_blocks=0):
     """Runs T steps on the GPU and in the oracle on identical inputs; returns both end states."""
     d = _lib()
     dev = torch.device("cuda:0")
     st = State(w, dev, align=align, byte_shift=byte_shift, v_init=v_init)
     eng = make_engine(d, w, st, post)
-    if ctas_per_sm:
-        eng.set_launch_shape(ctas_per_sm)
+    if max_blocks:
+        d.desloc_testing_set_max_blocks(eng.ctx, max_blocks)   # blocks stride over the chunks
     ox, ou = st.to_numpy(st.x), st.to_numpy(st.u)
     ov = st.to_numpy(st.v) if st.v is not None else None
     ocfg = oracle_cfg(w, oracle.FLAG_POST_AVERAGE if post else 0)
@@ -173,7 +173,7 @@ def test_mini_workloads_full_oracle(name):
     w = di.mini(di.WORKLOADS[name], T=40)
     if max(w.K) > 16:
         w = w.replace(K=tuple(max(1, k // 8) for k in w.K))
-    res = run_both(w, w.T, ctas_per_sm=0)
+    res = run_both(w, w.T)
     worst = check(res)
     assert res["counters"][0] == w.T
     assert sum(res["counters"][1:]) == sum(bin(m).count("1") for m in res["ref_masks"])
@@ -193,10 +193,13 @@ def test_mini_workloads_full_horizon_and_periods(name):
     print(name, w.T, worst)
 
 
-def test_persistent_grid_gives_identical_bits():
-    w = di.mini(di.WORKLOADS["cfg2_adam_135m"], T=12).replace(K=(2, 3, 4))
-    a = run_both(w, w.T, ctas_per_sm=0)
-    b = run_both(w, w.T, ctas_per_sm=2)
+@pytest.mark.parametrize("M", [1, 4, 8, 12])
+def test_striding_grid_gives_identical_bits(M):
+    """A grid smaller than the number of chunks (blocks stride over the rest) must give the same
+    bits as one block per chunk: the step, local and diagnostics kernels all take the loop."""
+    w = di.mini(di.WORKLOADS["cfg2_adam_135m"], T=12).replace(M=M, K=(2, 3, 4))
+    a = run_both(w, w.T)
+    b = run_both(w, w.T, max_blocks=3)
     for k in ("gx", "gu", "gv"):
         assert np.array_equal(a[k], b[k])
 
