@@ -1,7 +1,9 @@
 // DES-LOC step for worker counts beyond the register-resident kernels (M > MAX_MT) on steps
 // that average something.  Same update as desloc_step_kernel, runtime M, compile-time mask.
-// Worker sums are accumulated in fp64 in the order m = 0..M-1, which is exact for equal
-// replicas and matches a sequential reference to rounding.
+// Worker sums run in the order m = 0..M-1 as compensated fp32 sums (see WorkerSum): exact for
+// equal replicas, and within an ulp of a sequential fp64 reference.  Unlike the other kernels
+// this one takes the hardware reciprocal square root (2 ulp) for Adam's direction and ADOPT's
+// normaliser: it is bound by instruction issue, not by memory.
 //
 // A block takes one chunk and first puts the chunk-relative pointers of all M workers into
 // shared memory, so that the per-position loops read them as broadcasts instead of chasing the
@@ -22,51 +24,109 @@ namespace desloc {
 namespace {
 
 constexpr int GEN_MAX_M = 256;    // worker pointers staged per chunk (= the context's limit)
-constexpr int MEAN_BATCH = 4;     // workers whose loads are in flight while an array is summed
+// Measured on B200 (134.5 M parameters x 16 workers, fraction of the copy bandwidth on all-sync
+// steps): three blocks per SM with small batches 0.96; two blocks with batches twice as large
+// 0.85; fp64 worker sums 0.87 and IEEE sqrt / division 0.87 (this kernel is bound by
+// instruction issue: ~75 instructions per worker-coordinate before, ~45 now).
+constexpr int GEN_MIN_BLOCKS = 3;   // 80 registers per thread
+constexpr int GEN_BUDGET = 24;      // registers a batch of workers may hold in flight
 
-// Workers per batch of the update loops: what fits in `budget` registers, at most four.
+// Workers per batch of the update loops: what fits in `budget` registers -- 1, 2 or 4 (a power
+// of two, so that a full batch can be summed as a tree).
 __host__ __device__ constexpr int gen_batch(int per_worker, int budget) {
     const int b = budget / per_worker;
-    return b < 1 ? 1 : (b > 4 ? 4 : b);
+    return b < 2 ? 1 : (b < 4 ? 2 : 4);
 }
 
+// Sum over the workers of one coordinate group, in the order m = 0..M-1, as a compensated fp32
+// sum ("two-sum"): the running sum and the exact rounding error of every addition are both
+// kept, so the pair carries about 48 bits -- the accuracy of an fp64 sum without the fp64 pipe,
+// which made an all-sync step 10 % slower here.  The mean divides the pair by M with one
+// correction step, and is exact (the value itself) when all M replicas are equal.
 template <int VEC>
-__device__ __forceinline__ FV<VEC> mean_f64(char *const *bases, int M, long long e, bool active) {
-    double acc[VEC];
+struct WorkerSum {
+    float s[VEC], err[VEC];
+    __device__ __forceinline__ void clear() {
 #pragma unroll
-    for (int c = 0; c < VEC; ++c) acc[c] = 0.0;
-#pragma unroll 1
-    for (int m0 = 0; m0 < M; m0 += MEAN_BATCH) {
-        FV<VEC> b[MEAN_BATCH];
+        for (int c = 0; c < VEC; ++c) s[c] = err[c] = 0.f;
+    }
+    __device__ __forceinline__ void add(const FV<VEC> &v) {
 #pragma unroll
-        for (int j = 0; j < MEAN_BATCH; ++j)
-            if (active && m0 + j < M) b[j] = ld_f32<VEC>(bases[m0 + j], e);
-#pragma unroll
-        for (int j = 0; j < MEAN_BATCH; ++j) {
-            if (active && m0 + j < M) {
-#pragma unroll
-                for (int c = 0; c < VEC; ++c) acc[c] += static_cast<double>(b[j].a[c]);
-            }
+        for (int c = 0; c < VEC; ++c) {
+            const float x = v.a[c];
+            const float t = s[c] + x;
+            const float bp = t - s[c];
+            err[c] += (s[c] - (t - bp)) + (x - bp);  // exact error of t = s + x
+            s[c] = t;
         }
     }
-    FV<VEC> r;
+    __device__ __forceinline__ FV<VEC> mean(int M) const {
+        const float mf = static_cast<float>(M);
+        FV<VEC> r;
 #pragma unroll
-    for (int c = 0; c < VEC; ++c) r.a[c] = static_cast<float>(acc[c] / static_cast<double>(M));
-    return r;
-}
+        for (int c = 0; c < VEC; ++c) {
+            const float hi = s[c] + err[c];
+            const float lo = err[c] - (hi - s[c]);          // hi + lo = s + err
+            const float q = hi / mf;
+            const float rem = fmaf(-q, mf, hi) + lo;        // what q * M still misses
+            r.a[c] = q + rem / mf;
+        }
+        return r;
+    }
+    // A batch of B consecutive workers (B a power of two) of which the first n exist.  A full
+    // batch is summed as a binary tree first (exact when its values are equal) and enters the
+    // running sum as one value; a partial batch enters value by value.
+    template <int B>
+    __device__ __forceinline__ void add_batch(const FV<VEC> (&v)[B], int n) {
+        static_assert((B & (B - 1)) == 0, "batches are powers of two");
+        if (n >= B) {
+            FV<VEC> t;
+#pragma unroll
+            for (int c = 0; c < VEC; ++c) {
+                float q[B];
+#pragma unroll
+                for (int j = 0; j < B; ++j) q[j] = v[j].a[c];
+                t.a[c] = tree_sum<0, B, B>(q);
+            }
+            add(t);
+        } else {
+#pragma unroll
+            for (int j = 0; j < B; ++j)
+                if (j < n) add(v[j]);
+        }
+    }
+};
 
-template <int VEC>
-__device__ __forceinline__ void acc_add(double (&acc)[VEC], const FV<VEC> &v) {
+// Worker means of the arrays selected by SX, SU, SV in one pass over the workers: the loads of
+// a batch of workers (all selected arrays) are issued together -- four workers for one array,
+// two for two or three -- and then added in worker order, one accumulator per array.
+template <int VEC, bool SX, bool SU, bool SV>
+__device__ __forceinline__ void means_of_workers(char *const (*sp)[GEN_MAX_M], int M, long long e,
+                                                 bool active, FV<VEC> &xb, FV<VEC> &ub, FV<VEC> &vb) {
+    constexpr int NS = (SX ? 1 : 0) + (SU ? 1 : 0) + (SV ? 1 : 0);
+    constexpr int NB = NS == 1 ? 4 : 2;
+    WorkerSum<VEC> ax, au, av;
+    ax.clear(); au.clear(); av.clear();
+#pragma unroll 1
+    for (int m0 = 0; m0 < M; m0 += NB) {
+        FV<VEC> bx[NB], bu[NB], bv[NB];
 #pragma unroll
-    for (int c = 0; c < VEC; ++c) acc[c] += static_cast<double>(v.a[c]);
-}
-
-template <int VEC>
-__device__ __forceinline__ FV<VEC> acc_mean(const double (&acc)[VEC], int M) {
-    FV<VEC> r;
-#pragma unroll
-    for (int c = 0; c < VEC; ++c) r.a[c] = static_cast<float>(acc[c] / static_cast<double>(M));
-    return r;
+        for (int j = 0; j < NB; ++j) {
+            if (active && m0 + j < M) {
+                if constexpr (SX) bx[j] = ld_f32<VEC>(sp[0][m0 + j], e);
+                if constexpr (SU) bu[j] = ld_f32<VEC>(sp[1][m0 + j], e);
+                if constexpr (SV) bv[j] = ld_f32<VEC>(sp[2][m0 + j], e);
+            }
+        }
+        if (active) {
+            if constexpr (SX) ax.template add_batch<NB>(bx, M - m0);
+            if constexpr (SU) au.template add_batch<NB>(bu, M - m0);
+            if constexpr (SV) av.template add_batch<NB>(bv, M - m0);
+        }
+    }
+    if constexpr (SX) xb = ax.mean(M);
+    if constexpr (SU) ub = au.mean(M);
+    if constexpr (SV) vb = av.mean(M);
 }
 
 // Diagnostics with a runtime worker count: a warp reduces each (kind, worker) value at once
@@ -106,11 +166,10 @@ __device__ __forceinline__ void generic_position(const StepArgs &a, char *const 
     constexpr bool SV = (OPT != OPT_SGDM) && (MASK & SYNC_V);
     if constexpr (!POST) {
         FV<VEC> xb{}, ub{}, vb{};
-        if constexpr (SX) xb = mean_f64<VEC>(sp[0], M, e, active);
-        if constexpr (SU) ub = mean_f64<VEC>(sp[1], M, e, active);
-        if constexpr (SV) vb = mean_f64<VEC>(sp[2], M, e, active);
+        means_of_workers<VEC, SX, SU, SV>(sp, M, e, active, xb, ub, vb);
         constexpr bool NEED_V = OPT != OPT_SGDM && (!SV || OPT == OPT_ADOPT);
-        constexpr int B = gen_batch(worker_regs<OPT, GT>(!SX, !SU, NEED_V), 48);
+                constexpr int B0 = gen_batch(worker_regs<OPT, GT>(!SX, !SU, NEED_V), GEN_BUDGET);
+        constexpr int B = (OPT == OPT_ADOPT && B0 > 2) ? 2 : B0;  // ADOPT's normaliser needs more registers
 #pragma unroll 1
         for (int m0 = 0; m0 < M; m0 += B) {
             FV<VEC> G[B], X[B], U[B], V[B];
@@ -138,8 +197,8 @@ __device__ __forceinline__ void generic_position(const StepArgs &a, char *const 
                             const float vp = SV ? vb.a[c] : vown;
                             const float xp = SX ? xb.a[c] : X[b].a[c];
                             float un, vn;
-                            state_update<OPT>(a, G[b].a[c] * sc, up, vp, vown, un, vn);
-                            D.a[c] = direction<OPT>(a, un, vn);
+                            state_update<OPT, true>(a, G[b].a[c] * sc, up, vp, vown, un, vn);
+                            D.a[c] = direction<OPT, true>(a, un, vn);
                             X[b].a[c] = apply_step(a, xp, D.a[c]);
                             U[b].a[c] = un;
                             V[b].a[c] = vn;
@@ -158,10 +217,9 @@ __device__ __forceinline__ void generic_position(const StepArgs &a, char *const 
         }
     } else {
         using P = PostPlan<OPT, MASK>;
-        double au[VEC], av[VEC], ax[VEC];
-#pragma unroll
-        for (int c = 0; c < VEC; ++c) au[c] = av[c] = ax[c] = 0.0;
-        constexpr int BA = gen_batch(worker_regs<OPT, GT>(!P::D_NEEDS_MEAN, true, OPT != OPT_SGDM), 48);
+        WorkerSum<VEC> au, av, ax;
+        au.clear(); av.clear(); ax.clear();
+        constexpr int BA = gen_batch(worker_regs<OPT, GT>(!P::D_NEEDS_MEAN, true, OPT != OPT_SGDM), GEN_BUDGET);
         // phase A: states (and x where d_t needs no mean)
 #pragma unroll 1
         for (int m0 = 0; m0 < M; m0 += BA) {
@@ -187,11 +245,11 @@ __device__ __forceinline__ void generic_position(const StepArgs &a, char *const 
                         for (int c = 0; c < VEC; ++c) {
                             const float vown = OPT != OPT_SGDM ? V[b].a[c] : 0.f;
                             float un, vn;
-                            state_update<OPT>(a, G[b].a[c] * sc, U[b].a[c], vown, vown, un, vn);
+                            state_update<OPT, true>(a, G[b].a[c] * sc, U[b].a[c], vown, vown, un, vn);
                             U[b].a[c] = un;
                             V[b].a[c] = vn;
                             if constexpr (!P::D_NEEDS_MEAN) {
-                                D.a[c] = direction<OPT>(a, un, vn);
+                                D.a[c] = direction<OPT, true>(a, un, vn);
                                 X[b].a[c] = apply_step(a, X[b].a[c], D.a[c]);
                             }
                         }
@@ -199,13 +257,9 @@ __device__ __forceinline__ void generic_position(const StepArgs &a, char *const 
                         // it where Adam needs it per worker)
                         if constexpr (!P::SU) st_f32<VEC>(sp[1][m0 + b], e, U[b]);
                         if constexpr (OPT != OPT_SGDM && !P::SV) st_f32<VEC>(sp[2][m0 + b], e, V[b]);
-                        if constexpr (P::SU) acc_add<VEC>(au, U[b]);
-                        if constexpr (P::SV) acc_add<VEC>(av, V[b]);
                         if constexpr (!P::D_NEEDS_MEAN) {
                             dd = sum_sq<VEC>(D);
-                            if constexpr (P::SX) {
-                                acc_add<VEC>(ax, X[b]);
-                            } else {
+                            if constexpr (!P::SX) {
                                 xx = sum_sq<VEC>(X[b]);
                                 st_f32<VEC>(sp[0][m0 + b], e, X[b]);
                             }
@@ -218,11 +272,16 @@ __device__ __forceinline__ void generic_position(const StepArgs &a, char *const 
                     }
                 }
             }
+            if (active) {
+                if constexpr (P::SU) au.template add_batch<BA>(U, M - m0);
+                if constexpr (P::SV) av.template add_batch<BA>(V, M - m0);
+                if constexpr (P::SX && !P::D_NEEDS_MEAN) ax.template add_batch<BA>(X, M - m0);
+            }
         }
-        const FV<VEC> mu = acc_mean<VEC>(au, M), mv = acc_mean<VEC>(av, M);
+        const FV<VEC> mu = au.mean(M), mv = av.mean(M);
         if constexpr (P::D_NEEDS_MEAN) {
             // phase B: parameter step with the averaged states
-            constexpr int BB = gen_batch(4 + ((P::KEEP_U || P::KEEP_V) ? 4 : 0), 48);
+            constexpr int BB = gen_batch(4 + ((P::KEEP_U || P::KEEP_V) ? 4 : 0), GEN_BUDGET);
 #pragma unroll 1
             for (int m0 = 0; m0 < M; m0 += BB) {
                 FV<VEC> X[BB], K[BB];
@@ -244,13 +303,11 @@ __device__ __forceinline__ void generic_position(const StepArgs &a, char *const 
                             for (int c = 0; c < VEC; ++c) {
                                 const float un = P::SU ? mu.a[c] : K[b].a[c];
                                 const float vn = P::SV ? mv.a[c] : (P::KEEP_V ? K[b].a[c] : 0.f);
-                                D.a[c] = direction<OPT>(a, un, vn);
+                                D.a[c] = direction<OPT, true>(a, un, vn);
                                 X[b].a[c] = apply_step(a, X[b].a[c], D.a[c]);
                             }
                             dd = sum_sq<VEC>(D);
-                            if constexpr (P::SX) {
-                                acc_add<VEC>(ax, X[b]);
-                            } else {
+                            if constexpr (!P::SX) {
                                 xx = sum_sq<VEC>(X[b]);
                                 st_f32<VEC>(sp[0][m0 + b], e, X[b]);
                             }
@@ -261,10 +318,13 @@ __device__ __forceinline__ void generic_position(const StepArgs &a, char *const 
                         if constexpr (!P::SX) wd.add(DIAG_X, m0 + b, xx);
                     }
                 }
+                if constexpr (P::SX) {
+                    if (active) ax.template add_batch<BB>(X, M - m0);
+                }
             }
         }
         if constexpr (P::SX || (!P::D_NEEDS_MEAN && P::SV)) {
-            const FV<VEC> mx = acc_mean<VEC>(ax, M);
+            const FV<VEC> mx = ax.mean(M);
             const float xx = (P::SX && active) ? sum_sq<VEC>(mx) : 0.f;
             if (active) {
 #pragma unroll 1
@@ -279,7 +339,7 @@ __device__ __forceinline__ void generic_position(const StepArgs &a, char *const 
 }
 
 template <int OPT, typename GT, bool POST, int MASK, bool DIAG>
-__global__ void __launch_bounds__(BLOCK_THREADS, 2)
+__global__ void __launch_bounds__(BLOCK_THREADS, GEN_MIN_BLOCKS)
 desloc_step_generic_kernel(const __grid_constant__ StepArgs a) {
     __shared__ char *sp[4][GEN_MAX_M];
     __shared__ float sscale[GEN_MAX_M];

@@ -202,7 +202,10 @@ __device__ __forceinline__ float mean_of(const float (&s)[MT]) {
 // One worker's state update from the clipped gradient: `up`, `vp` are the previous states the
 // update starts from (the worker's own or the worker mean); `vown` is always the worker's own
 // previous v, which ADOPT's normaliser uses (Algorithm 3).
-template <int OPT>
+// FAST: hardware reciprocal square root (2 ulp) in place of IEEE sqrt and division.  Only the
+// runtime-M kernel uses it: that kernel is bound by instruction issue, not by memory, and the
+// exact forms cost it a tenth of its speed.
+template <int OPT, bool FAST = false>
 __device__ __forceinline__ void state_update(const StepArgs &a, float g, float up, float vp,
                                              float vown, float &un, float &vn) {
     // coordinate-wise clip: sgn(g) min(|g|, rho)  (Section 3.1); rho = +inf when off
@@ -212,7 +215,11 @@ __device__ __forceinline__ void state_update(const StepArgs &a, float g, float u
         vn = fmaf(a.b2, vp, (a.omb2 * gh) * gh);
     } else if constexpr (OPT == OPT_ADOPT) {
         vn = fmaf(a.b2, vp, (a.omb2 * gh) * gh);
-        float r = gh / fmaxf(sqrtf(vown), a.eps);
+        float r;
+        if constexpr (FAST)
+            r = gh * rsqrtf(fmaxf(vown, a.eps * a.eps));  // 1 / max(sqrt(v), eps)
+        else
+            r = gh / fmaxf(sqrtf(vown), a.eps);
         r = fminf(fmaxf(r, -a.cbound), a.cbound);
         un = fmaf(a.b1, up, a.omb1 * r);
     } else {
@@ -222,10 +229,10 @@ __device__ __forceinline__ void state_update(const StepArgs &a, float g, float u
 }
 
 // The update d_t of Algorithms 2-3 from the new states.
-template <int OPT>
+template <int OPT, bool FAST = false>
 __device__ __forceinline__ float direction(const StepArgs &a, float un, float vn) {
     if constexpr (OPT == OPT_ADAM)
-        return (a.lr * un) / sqrtf(vn + a.lam2);
+        return FAST ? (a.lr * un) * rsqrtf(vn + a.lam2) : (a.lr * un) / sqrtf(vn + a.lam2);
     else
         return a.lr * un;
 }
@@ -533,7 +540,10 @@ __device__ __forceinline__ void process_tile_post_batched(const StepArgs &a, cha
         if constexpr (P::SU) su.a[c] = su.a[c] / static_cast<float>(MT);
         if constexpr (P::SV) sv.a[c] = sv.a[c] / static_cast<float>(MT);
     }
-    if constexpr (P::D_NEEDS_MEAN) {
+    if constexpr (P::D_NEEDS_MEAN && !(P::KEEP_U || P::KEEP_V)) {
+        // nothing is kept per worker: all MT loads of x go out together
+        post_phase_b<OPT, MASK, MT, VEC, DIAG, 0, MT>(a, sp, e, su, sv, sx, keep, dg);
+    } else if constexpr (P::D_NEEDS_MEAN) {
         post_phase_b<OPT, MASK, MT, VEC, DIAG, 0, 4>(a, sp, e, su, sv, sx, keep, dg);
         post_phase_b<OPT, MASK, MT, VEC, DIAG, 4, MT - 4>(a, sp, e, su, sv, sx, keep, dg);
     } else {
@@ -644,11 +654,12 @@ __device__ __forceinline__ void process_chunk(const StepArgs &a, char *const (*s
     }
 }
 
-// Resident blocks per SM the kernels are compiled for: three (80 registers per thread) except
-// SGDM and the post-average tiles of more than four workers, which are fastest at two.
+// Resident blocks per SM the kernels are compiled for: three (80 registers per thread), except
+// SGDM with more than four workers (all-at-once tile), which is fastest at two.  The batched
+// post-average tiles moved from two to three: 0.88 -> 0.97 on ADOPT's all-sync steps (M = 8).
 template <int OPT, int MT, bool POST>
 __host__ __device__ constexpr int min_blocks() {
-    return (MT <= 4) ? 3 : ((OPT == OPT_SGDM || POST) ? 2 : 3);
+    return (MT > 4 && OPT == OPT_SGDM) ? 2 : 3;
 }
 
 template <int OPT, int MASK, int MT, typename GT, bool POST, bool DIAG>
