@@ -8,9 +8,10 @@
  *
  * This library keeps all M worker replicas in ONE GPU's memory.  One call to
  * desloc_step() runs one step t of Algorithm 1 for all workers: a single
- * memory-bound kernel reads g, x, u, v of every replica once, clips the
- * gradient, averages the arrays whose period divides t in registers (a fixed
- * summation tree over m), applies the per-worker update and writes x, u, v back.
+ * memory-bound kernel brings g, x, u, v of every replica on chip once (tile by
+ * tile, with bulk asynchronous copies), clips the gradient, averages the arrays
+ * whose period divides t (a fixed summation tree over m), applies the
+ * per-worker update and writes x, u, v back.
  * A sync step therefore moves the same bytes as a local step; there is no
  * separate averaging pass and no collective.
  *
@@ -73,7 +74,10 @@ typedef enum {
     DESLOC_E_INVALID = -3, /* unknown optimizer / dtype / flag, or a flag the optimizer lacks */
     DESLOC_E_NOMEM = -4,   /* host or device allocation failed */
     DESLOC_E_CUDA = -5,    /* a CUDA call failed; see desloc_last_cuda_error() */
-    DESLOC_E_TOO_LARGE = -6 /* desloc_step_static(): the problem exceeds the fixed scratch */
+    DESLOC_E_TOO_LARGE = -6, /* desloc_step_static(): the problem exceeds the fixed scratch */
+    DESLOC_E_DEVICE_WAIT = -7 /* a thread block of an earlier step gave up waiting for its data
+                                 (every wait on the device is bounded): that step is incomplete and
+                                 the state undefined; every later step call returns this status */
 } desloc_status;
 
 /* The "Require" block of Algorithms 1-3: everything fixed for a run.  Plain data, copied
@@ -255,8 +259,7 @@ DESLOC_API int desloc_destroy(desloc_ctx *ctx);
    distributed run of the same schedule would pay; Section 5.1 "Metrics"). */
 DESLOC_API int desloc_get_counters(const desloc_ctx *ctx, int64_t out[4]);
 
-/* Kernels launched by this context so far (one per step on the main path, one thread block
-   per chunk). */
+/* Kernels launched by this context so far (one per step on the main path). */
 DESLOC_API int64_t desloc_get_launch_count(const desloc_ctx *ctx);
 
 /*
@@ -269,9 +272,10 @@ DESLOC_API int64_t desloc_get_launch_count(const desloc_ctx *ctx);
 DESLOC_API int64_t desloc_plan_chunks(const int64_t *numel, int32_t num_tensors, int64_t chunk_elems,
                            int64_t *out, int64_t cap);
 
-/* Elements per chunk used by contexts of this build (problems of fewer than 296 such chunks
-   are cut into chunks a quarter of this size). */
-DESLOC_API int64_t desloc_chunk_elems(void);
+/* Elements per chunk (the tile one thread block works on, for all workers) of a context with M
+   workers: 1024 for M <= 2 and M > 8, 512 for M = 3, 4, 256 for M = 5..8.  DESLOC_E_RANGE for an
+   M outside 1..DESLOC_MAX_M. */
+DESLOC_API int64_t desloc_chunk_elems(int32_t M);
 
 /*
  * desloc_step_static(): one step for callers that cannot allocate.  (The paper has no
@@ -283,13 +287,13 @@ DESLOC_API int64_t desloc_chunk_elems(void);
  * to give memory back), and a latency-critical loop cannot afford the device-wide
  * synchronisation that cudaMalloc and cudaFree bring.  This entry point needs no context and
  * calls no cudaMalloc, cudaFree, cudaMallocHost or any other allocating routine: its tables
- * go into a fixed array inside the library image, DESLOC_STATIC_SCRATCH_BYTES (about 320 KB)
- * of device memory per GPU, held until the process exits.
+ * go into a fixed array inside the library image, DESLOC_STATIC_SCRATCH_BYTES (576 KB) of
+ * device memory per GPU, held until the process exits.
  *
  * Limits: M * num_tensors <= DESLOC_STATIC_MAX_POINTERS, M <= 8, and at most
- * DESLOC_STATIC_MAX_CHUNKS chunks (the chunk length is the one a context would use for the
- * same tensor list; every tensor starts a new chunk) -- up to 64 Mi parameters when tensors
- * are large.  Anything bigger returns DESLOC_E_TOO_LARGE and does nothing.
+ * DESLOC_STATIC_MAX_CHUNKS chunks of desloc_chunk_elems(M) elements (every tensor starts a new
+ * chunk) -- up to 32 Mi parameters for M <= 2, 16 Mi for M = 3, 4 and 8 Mi for M = 5..8 when
+ * tensors are large.  Anything bigger returns DESLOC_E_TOO_LARGE and does nothing.
  *
  * Arguments as for desloc_create() + desloc_step(): cfg, the host arrays x, u, v, grads of
  * M*num_tensors DEVICE pointers (v may be NULL for SGDM), the step t, eta_t, the ADOPT bound,
@@ -300,7 +304,7 @@ DESLOC_API int64_t desloc_chunk_elems(void);
  * Set-up.  The first call on each device looks up the device address of the array
  * (cudaGetSymbolAddress, with that device current).  With the CUDA runtime's lazy module
  * loading that look-up is also the moment the runtime loads the module and reserves the
- * array's 320 KB on that GPU: make the first call at start-up -- before a framework's pool has
+ * array's 576 KB on that GPU: make the first call at start-up -- before a framework's pool has
  * grown to fill the device, where it could fail with DESLOC_E_CUDA, and before any stream
  * capture begins.  The address is remembered per device for the life of the process and does
  * not survive a cudaDeviceReset().
@@ -321,7 +325,7 @@ DESLOC_API int64_t desloc_chunk_elems(void);
  * caller; calls issued one after the other on the same stream are safe.
  */
 #define DESLOC_STATIC_MAX_POINTERS 2048
-#define DESLOC_STATIC_MAX_CHUNKS 16384
+#define DESLOC_STATIC_MAX_CHUNKS 32768
 #define DESLOC_STATIC_SCRATCH_BYTES (DESLOC_STATIC_MAX_CHUNKS * 16 + 4 * DESLOC_STATIC_MAX_POINTERS * 8)
 DESLOC_API int desloc_step_static(const desloc_config *cfg, float *const *x, float *const *u,
                                   float *const *v, const void *const *grads, int64_t t,

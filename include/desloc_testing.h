@@ -20,6 +20,15 @@ extern "C" {
  */
 DESLOC_API int desloc_testing_set_max_blocks(desloc_ctx *ctx, int64_t max_blocks);
 
+/*
+ * How often a thread block polls for its tile's copies before it gives up (default: about four
+ * million polls).  polls = 0 makes every block give up at once: the step then stores nothing,
+ * the blocks still let their copies land before they leave, and every later step call returns
+ * DESLOC_E_DEVICE_WAIT -- the way the tests exercise the bounded-wait path without hanging or
+ * faulting anything.  A negative value restores the default and clears the recorded failure.
+ */
+DESLOC_API int desloc_testing_set_wait_limit(desloc_ctx *ctx, int32_t polls);
+
 #ifdef __cplusplus
 }
 #endif

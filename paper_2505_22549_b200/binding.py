@@ -21,7 +21,8 @@ DESLOC_FLAG_ADOPT_NORM_CLIP, DESLOC_FLAG_POST_AVERAGE = 1, 2
 DESLOC_OK, DESLOC_E_NULL, DESLOC_E_RANGE, DESLOC_E_INVALID, DESLOC_E_NOMEM, DESLOC_E_CUDA = \
     0, -1, -2, -3, -4, -5
 DESLOC_E_TOO_LARGE = -6
-DESLOC_STATIC_MAX_POINTERS, DESLOC_STATIC_MAX_CHUNKS = 2048, 16384
+DESLOC_E_DEVICE_WAIT = -7
+DESLOC_STATIC_MAX_POINTERS, DESLOC_STATIC_MAX_CHUNKS = 2048, 32768
 DESLOC_MAX_M = 256
 
 OPT_BY_NAME = {"adam": DESLOC_ADAM, "adopt": DESLOC_ADOPT, "sgdm": DESLOC_SGDM}
@@ -106,12 +107,14 @@ _lib.desloc_get_diag_norms.argtypes = [_P, ctypes.POINTER(ctypes.c_float),
                                        ctypes.POINTER(ctypes.c_float), _P]
 _lib.desloc_testing_set_max_blocks.restype = ctypes.c_int
 _lib.desloc_testing_set_max_blocks.argtypes = [_P, ctypes.c_int64]
+_lib.desloc_testing_set_wait_limit.restype = ctypes.c_int
+_lib.desloc_testing_set_wait_limit.argtypes = [_P, ctypes.c_int32]
 _lib.desloc_plan_chunks.restype = ctypes.c_int64
 _lib.desloc_plan_chunks.argtypes = [ctypes.POINTER(ctypes.c_int64), ctypes.c_int32,
                                     ctypes.c_int64, ctypes.POINTER(ctypes.c_int64),
                                     ctypes.c_int64]
 _lib.desloc_chunk_elems.restype = ctypes.c_int64
-_lib.desloc_chunk_elems.argtypes = []
+_lib.desloc_chunk_elems.argtypes = [ctypes.c_int32]
 _lib.desloc_strerror.restype = ctypes.c_char_p
 _lib.desloc_strerror.argtypes = [ctypes.c_int]
 _lib.desloc_last_cuda_error.restype = ctypes.c_int
@@ -303,8 +306,20 @@ def desloc_testing_set_max_blocks(ctx: int, max_blocks: int) -> None:
         raise DeslocError(rc, "desloc_testing_set_max_blocks")
 
 
-def desloc_chunk_elems() -> int:
-    return int(_lib.desloc_chunk_elems())
+def desloc_chunk_elems(M: int) -> int:
+    """Elements per chunk (tile) of a context with M workers."""
+    n = int(_lib.desloc_chunk_elems(int(M)))
+    if n < 0:
+        raise DeslocError(n, "desloc_chunk_elems")
+    return n
+
+
+def desloc_testing_set_wait_limit(ctx: int, polls: int) -> None:
+    """Test hook (include/desloc_testing.h): bound on a block's wait for its tile; negative =
+    default, and clears a recorded failure."""
+    rc = _lib.desloc_testing_set_wait_limit(ctx, int(polls))
+    if rc != DESLOC_OK:
+        raise DeslocError(rc, "desloc_testing_set_wait_limit")
 
 
 def desloc_plan_chunks(numel: Sequence[int], chunk_elems: int, cap: Optional[int] = None):

@@ -57,11 +57,22 @@ struct Slot {
     bool in_flight = false;
 };
 
-// Everything whose size depends on the worker count M (re-made by desloc_set_workers).
+// desloc_step_host: tensor groups whose copies and kernels are pipelined
+struct HostGroup {
+    int32_t k0, k1;   // tensors [k0, k1)
+    int64_t c0, c1;   // tiles   [c0, c1)
+};
+
+// Everything that depends on the worker count M (re-made by desloc_set_workers): the pointer
+// tables, the tile plan (the tile length is a function of M) and the scratch sized by either.
 struct WorkerRes {
+    desloc::Chunk *d_chunks = nullptr;   // tiles of the step kernels
+    int64_t nchunks = 0;
+    long long *d_tstart = nullptr;       // [num_tensors + 1] first tile of every tensor
+    std::vector<HostGroup> groups;
     void **d_tables = nullptr;  // [3][nptr] x, u, v
     Slot slots[kSlots];
-    float *d_partial = nullptr;  // reductions: partial sums [2][M][nchunks]
+    float *d_partial = nullptr;  // reductions: partial sums [2][M][nrchunks]
     float *d_norms = nullptr;    // [3][M]: gradient norms, clip factors, relative change
     void **h_snap = nullptr;     // pinned pointer table for desloc_rel_change
     void **d_snap = nullptr;
@@ -77,6 +88,8 @@ void free_worker_res(WorkerRes &r) {
         if (s.dev) cudaFree(s.dev);
         s = Slot();
     }
+    if (r.d_chunks) cudaFree(r.d_chunks);
+    if (r.d_tstart) cudaFree(r.d_tstart);
     if (r.d_tables) cudaFree(r.d_tables);
     if (r.d_partial) cudaFree(r.d_partial);
     if (r.d_norms) cudaFree(r.d_norms);
@@ -88,9 +101,43 @@ void free_worker_res(WorkerRes &r) {
     r = WorkerRes();
 }
 
-// Allocates and fills the M-dependent resources; the device must be current.
-cudaError_t make_worker_res(WorkerRes &r, int M, int num_tensors, int64_t nchunks, bool has_v,
-                            float *const *x, float *const *u, float *const *v) {
+// Allocates and fills the M-dependent resources; the device must be current.  May throw
+// std::bad_alloc (host vectors).
+cudaError_t make_worker_res(WorkerRes &r, int M, const int64_t *numel, int num_tensors, int64_t total,
+                            int64_t nrchunks, bool has_v, float *const *x, float *const *u,
+                            float *const *v) {
+    // tile plan for this worker count
+    const int64_t chunk_elems = desloc::chunk_elems_for(M);
+    const int64_t nchunks = desloc::count_chunks(numel, num_tensors, chunk_elems);
+    std::vector<desloc::Chunk> chunks(static_cast<size_t>(nchunks));
+    desloc::fill_chunks(numel, num_tensors, chunk_elems, chunks.data());
+    std::vector<long long> tstart(static_cast<size_t>(num_tensors) + 1, 0);
+    r.groups.clear();
+    {
+        // tensor groups of about equal size for desloc_step_host
+        int64_t acc = 0, c0 = 0;
+        int32_t k0 = 0;
+        for (int32_t k = 0; k < num_tensors; ++k) {
+            tstart[k + 1] = tstart[k] + (numel[k] + chunk_elems - 1) / chunk_elems;
+            acc += numel[k];
+            const int done_groups = static_cast<int>(r.groups.size());
+            const bool last = k == num_tensors - 1;
+            if (last || (done_groups < kHostGroups - 1 && acc * kHostGroups >= total * (done_groups + 1))) {
+                r.groups.push_back({k0, k + 1, c0, tstart[k + 1]});
+                k0 = k + 1;
+                c0 = tstart[k + 1];
+            }
+        }
+    }
+    r.nchunks = nchunks;
+    cudaError_t e0 = cudaMalloc(&r.d_chunks, chunks.size() * sizeof(desloc::Chunk));
+    if (e0 == cudaSuccess)
+        e0 = cudaMemcpy(r.d_chunks, chunks.data(), chunks.size() * sizeof(desloc::Chunk), cudaMemcpyHostToDevice);
+    if (e0 == cudaSuccess) e0 = cudaMalloc(&r.d_tstart, tstart.size() * sizeof(long long));
+    if (e0 == cudaSuccess)
+        e0 = cudaMemcpy(r.d_tstart, tstart.data(), tstart.size() * sizeof(long long), cudaMemcpyHostToDevice);
+    if (e0 != cudaSuccess) return e0;
+
     const int64_t nptr = static_cast<int64_t>(M) * num_tensors;
     std::vector<void *> tables(static_cast<size_t>(3 * nptr), nullptr);
     for (int64_t i = 0; i < nptr; ++i) {
@@ -101,7 +148,7 @@ cudaError_t make_worker_res(WorkerRes &r, int M, int num_tensors, int64_t nchunk
     cudaError_t e = cudaMalloc(&r.d_tables, tables.size() * sizeof(void *));
     if (e == cudaSuccess)
         e = cudaMemcpy(r.d_tables, tables.data(), tables.size() * sizeof(void *), cudaMemcpyHostToDevice);
-    const size_t npart = static_cast<size_t>(2) * M * static_cast<size_t>(nchunks);
+    const size_t npart = static_cast<size_t>(2) * M * static_cast<size_t>(nrchunks);
     if (e == cudaSuccess) e = cudaMalloc(&r.d_partial, npart * sizeof(float));
     if (e == cudaSuccess) e = cudaMalloc(&r.d_norms, static_cast<size_t>(3) * M * sizeof(float));
     if (e == cudaSuccess) e = cudaMemset(r.d_norms, 0, static_cast<size_t>(3) * M * sizeof(float));
@@ -128,8 +175,11 @@ struct desloc_ctx {
     int device = 0;
     int64_t total_elems = 0;
     int64_t nptr = 0;  // M * num_tensors
-    desloc::Chunk *d_chunks = nullptr;
-    int64_t nchunks = 0;
+    desloc::Chunk *d_rchunks = nullptr;  // 4096-element chunks of the reduction kernels
+    int64_t nrchunks = 0;
+    int *h_err = nullptr;                // mapped pinned flag: a device-side wait ran out
+    int *d_err = nullptr;                // the same flag as the kernels address it
+    int wait_limit = desloc::DEFAULT_WAIT_LIMIT;
     WorkerRes res;
     int next_slot = 0;
     int cur_slot = -1;           // slot holding the table equal to last_grads
@@ -138,15 +188,8 @@ struct desloc_ctx {
     int64_t counters[4] = {0, 0, 0, 0};
     int64_t launches = 0;
     int last_cuda_error = 0;
-    long long *d_tstart = nullptr;  // [num_tensors + 1] first chunk of every tensor
     bool diag_valid = false;        // a diagnostics step has run since the workers last changed
     int64_t max_blocks = 0;         // test hook: cap on the grid (0 = one block per work item)
-    // desloc_step_host: tensor groups whose copies and kernels are pipelined
-    struct Group {
-        int32_t k0, k1;   // tensors [k0, k1)
-        int64_t c0, c1;   // chunks  [c0, c1)
-    };
-    std::vector<Group> groups;
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t ev_entry = nullptr;
     cudaEvent_t ev_group[kHostGroups] = {};
@@ -167,8 +210,8 @@ void free_ctx(desloc_ctx *ctx) {
     if (ctx->ev_entry) cudaEventDestroy(ctx->ev_entry);
     for (cudaEvent_t ev : ctx->ev_group)
         if (ev) cudaEventDestroy(ev);
-    if (ctx->d_chunks) cudaFree(ctx->d_chunks);
-    if (ctx->d_tstart) cudaFree(ctx->d_tstart);
+    if (ctx->d_rchunks) cudaFree(ctx->d_rchunks);
+    if (ctx->h_err) cudaFreeHost(ctx->h_err);
     delete ctx;
 }
 
@@ -212,6 +255,8 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
     if (rc != DESLOC_OK) return rc;
     for (int64_t i = 0; i < ctx->nptr; ++i)
         if (!grads[i]) return DESLOC_E_NULL;
+    // a block of an earlier step gave up waiting for its tile: that step is incomplete
+    if (*static_cast<volatile int *>(ctx->h_err) != 0) return DESLOC_E_DEVICE_WAIT;
 
     int dev_before = -1;
     cudaError_t e = cudaGetDevice(&dev_before);
@@ -251,7 +296,7 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
         }
         const float *d_gscale = nullptr;
         if (max_norm > 0.f) {
-            e = desloc::launch_grad_norms(ctx->d_chunks, ctx->nchunks,
+            e = desloc::launch_grad_norms(ctx->d_rchunks, ctx->nrchunks,
                                           reinterpret_cast<const void *const *>(d_g), c.num_tensors,
                                           c.M, c.grad_dtype == DESLOC_BF16, max_norm,
                                           ctx->res.d_partial, ctx->res.d_norms, ctx->res.d_norms + c.M, stream);
@@ -263,14 +308,14 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
             d_gscale = ctx->res.d_norms + c.M;
         }
 
-        const desloc::LaunchPlan plan = desloc::plan_launch(c, mask, ctx->nchunks, diag);
+        const desloc::LaunchPlan plan = desloc::plan_launch(c, mask, ctx->res.nchunks, diag);
         if (!plan.fn) {
             rc = DESLOC_E_INVALID;
             break;
         }
         desloc::StepArgs a{};
-        a.chunks = ctx->d_chunks;
-        a.nchunks = ctx->nchunks;
+        a.chunks = ctx->res.d_chunks;
+        a.nchunks = ctx->res.nchunks;
         a.x = reinterpret_cast<float *const *>(ctx->res.d_tables);
         a.u = reinterpret_cast<float *const *>(ctx->res.d_tables + ctx->nptr);
         a.v = reinterpret_cast<float *const *>(ctx->res.d_tables + 2 * ctx->nptr);
@@ -279,9 +324,11 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
             for (int64_t i = 0; i < ctx->nptr; ++i) a.g_inline[i] = grads[i];
         a.gscale = d_gscale;
         a.diag = diag ? ctx->res.d_diag : nullptr;
-        a.diag_stride = ctx->nchunks;
+        a.diag_stride = ctx->res.nchunks;
         a.diag_chunk0 = 0;
         desloc::fill_hyper(a, c, lr_t, clip_bound_t);
+        a.err = ctx->d_err;
+        a.wait_limit = ctx->wait_limit;
 
         void *params[] = {&a};
         const auto capped = [ctx](const desloc::LaunchPlan &lp) {
@@ -297,8 +344,8 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
             const size_t gsz = c.grad_dtype == DESLOC_BF16 ? 2 : 4;
             e = cudaEventRecord(ctx->ev_entry, stream);
             if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_entry, 0);
-            for (size_t gi = 0; gi < ctx->groups.size() && e == cudaSuccess; ++gi) {
-                const desloc_ctx::Group &grp = ctx->groups[gi];
+            for (size_t gi = 0; gi < ctx->res.groups.size() && e == cudaSuccess; ++gi) {
+                const HostGroup &grp = ctx->res.groups[gi];
                 for (int m = 0; m < c.M && e == cudaSuccess; ++m) {
                     // merge tensors that are adjacent on both sides into one copy
                     int32_t k = grp.k0;
@@ -323,7 +370,7 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
                 if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_group[gi], ctx->copy_stream);
                 if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->ev_group[gi], 0);
                 if (e != cudaSuccess) break;
-                a.chunks = ctx->d_chunks + grp.c0;
+                a.chunks = ctx->res.d_chunks + grp.c0;
                 a.nchunks = grp.c1 - grp.c0;
                 a.diag_chunk0 = grp.c0;
                 const desloc::LaunchPlan gp = desloc::plan_launch(c, mask, a.nchunks, diag);
@@ -364,7 +411,9 @@ uint32_t desloc_sync_mask(const desloc_config *cfg, int64_t t) {
     return mask_at(cfg, t);
 }
 
-int64_t desloc_chunk_elems(void) { return desloc::CHUNK_ELEMS; }
+int64_t desloc_chunk_elems(int32_t M) {
+    return (M < 1 || M > DESLOC_MAX_M) ? DESLOC_E_RANGE : desloc::chunk_elems_for(M);
+}
 
 int64_t desloc_plan_chunks(const int64_t *numel, int32_t num_tensors, int64_t chunk_elems,
                            int64_t *out, int64_t cap) {
@@ -403,25 +452,20 @@ int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *const *x, f
         if (!x[i] || !u[i]) return DESLOC_E_NULL;
         if (cfg->opt != DESLOC_SGDM && !v[i]) return DESLOC_E_NULL;
     }
-    const int64_t chunk_elems = desloc::chunk_elems_for(cfg->numel, cfg->num_tensors);
-    const int64_t nchunks = desloc::count_chunks(cfg->numel, cfg->num_tensors, chunk_elems);
-    // one thread block per chunk (or per worker and group of chunks): the grid must fit
-    if (nchunks > 0x7fffffffLL ||
-        (nchunks / desloc::LOCAL_SLOTS + 1) * static_cast<int64_t>(cfg->M) > 0x7fffffffLL)
+    const int64_t nrchunks = desloc::count_chunks(cfg->numel, cfg->num_tensors, desloc::REDUCE_CHUNK_ELEMS);
+    // one thread block per tile (per worker and tile when workers are separate items): the grid
+    // must fit for every worker count the context may be switched to
+    if (desloc::count_chunks(cfg->numel, cfg->num_tensors, 256) > 0x7fffffffLL / DESLOC_MAX_M)
         return DESLOC_E_RANGE;
 
     desloc_ctx *ctx = new (std::nothrow) desloc_ctx();
     if (!ctx) return DESLOC_E_NOMEM;
-    std::vector<desloc::Chunk> chunks;
-    std::vector<long long> tstart;
+    std::vector<desloc::Chunk> rchunks;
     try {
         ctx->numel.assign(cfg->numel, cfg->numel + cfg->num_tensors);
         ctx->last_grads.assign(static_cast<size_t>(nptr), nullptr);
-        chunks.resize(static_cast<size_t>(nchunks));
-        desloc::fill_chunks(cfg->numel, cfg->num_tensors, chunk_elems, chunks.data());
-        tstart.assign(static_cast<size_t>(cfg->num_tensors) + 1, 0);
-        for (int32_t k = 0; k < cfg->num_tensors; ++k)
-            tstart[k + 1] = tstart[k] + (cfg->numel[k] + chunk_elems - 1) / chunk_elems;
+        rchunks.resize(static_cast<size_t>(nrchunks));
+        desloc::fill_chunks(cfg->numel, cfg->num_tensors, desloc::REDUCE_CHUNK_ELEMS, rchunks.data());
     } catch (const std::bad_alloc &) {
         delete ctx;
         return DESLOC_E_NOMEM;
@@ -431,42 +475,27 @@ int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *const *x, f
     ctx->device = cuda_device;
     ctx->total_elems = total;
     ctx->nptr = nptr;
-    ctx->nchunks = nchunks;
+    ctx->nrchunks = nrchunks;
 
     int dev_before = -1;
     cudaError_t e = cudaGetDevice(&dev_before);
     if (e == cudaSuccess && dev_before != cuda_device) e = cudaSetDevice(cuda_device);
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_chunks, chunks.size() * sizeof(desloc::Chunk));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_rchunks, rchunks.size() * sizeof(desloc::Chunk));
     if (e == cudaSuccess)
-        e = cudaMemcpy(ctx->d_chunks, chunks.data(), chunks.size() * sizeof(desloc::Chunk),
+        e = cudaMemcpy(ctx->d_rchunks, rchunks.data(), rchunks.size() * sizeof(desloc::Chunk),
                        cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_tstart, tstart.size() * sizeof(long long));
-    if (e == cudaSuccess)
-        e = cudaMemcpy(ctx->d_tstart, tstart.data(), tstart.size() * sizeof(long long),
-                       cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaHostAlloc(reinterpret_cast<void **>(&ctx->h_err), sizeof(int), cudaHostAllocMapped);
+    if (e == cudaSuccess) {
+        *ctx->h_err = 0;
+        e = cudaHostGetDevicePointer(reinterpret_cast<void **>(&ctx->d_err), ctx->h_err, 0);
+    }
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_entry, cudaEventDisableTiming);
     for (int i = 0; i < kHostGroups && e == cudaSuccess; ++i)
         e = cudaEventCreateWithFlags(&ctx->ev_group[i], cudaEventDisableTiming);
     if (e == cudaSuccess) {
         try {
-            // tensor groups of about equal size for desloc_step_host
-            int64_t c = 0, acc = 0;
-            int32_t k0 = 0;
-            int64_t c0 = 0;
-            for (int32_t k = 0; k < cfg->num_tensors; ++k) {
-                c += (cfg->numel[k] + chunk_elems - 1) / chunk_elems;
-                acc += cfg->numel[k];
-                const int done_groups = static_cast<int>(ctx->groups.size());
-                const bool last = k == cfg->num_tensors - 1;
-                if (last || (done_groups < kHostGroups - 1 &&
-                             acc * kHostGroups >= total * (done_groups + 1))) {
-                    ctx->groups.push_back({k0, k + 1, c0, c});
-                    k0 = k + 1;
-                    c0 = c;
-                }
-            }
-            e = make_worker_res(ctx->res, cfg->M, cfg->num_tensors, ctx->nchunks,
+            e = make_worker_res(ctx->res, cfg->M, ctx->numel.data(), cfg->num_tensors, total, nrchunks,
                                 cfg->opt != DESLOC_SGDM, x, u, v);
         } catch (const std::bad_alloc &) {
             e = cudaErrorMemoryAllocation;
@@ -516,7 +545,7 @@ int desloc_get_diag_norms(desloc_ctx *ctx, float *per_tensor_out, float *total_o
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     const size_t rows = static_cast<size_t>(desloc::DIAG_KINDS) * c.M;
     float *d_per = ctx->res.d_diag_out, *d_tot = ctx->res.d_diag_out + rows * c.num_tensors;
-    e = desloc::launch_diag_norms(ctx->res.d_diag, ctx->nchunks, ctx->d_tstart, c.num_tensors, c.M,
+    e = desloc::launch_diag_norms(ctx->res.d_diag, ctx->res.nchunks, ctx->res.d_tstart, c.num_tensors, c.M,
                                   ctx->res.d_diag_sums, d_per, d_tot, st);
     if (e == cudaSuccess) {
         ctx->launches += 2;
@@ -603,7 +632,7 @@ int desloc_rel_change(desloc_ctx *ctx, int32_t array, const float *const *then, 
     float *d_out = ctx->res.d_norms + 2 * ctx->cfg.M;
     if (e == cudaSuccess)
         e = desloc::launch_rel_change(
-            ctx->d_chunks, ctx->nchunks,
+            ctx->d_rchunks, ctx->nrchunks,
             reinterpret_cast<const float *const *>(ctx->res.d_tables + array * ctx->nptr),
             reinterpret_cast<const float *const *>(ctx->res.d_snap), ctx->cfg.num_tensors, ctx->cfg.M,
             ctx->res.d_partial, d_out, st);
@@ -638,7 +667,7 @@ int desloc_set_workers(desloc_ctx *ctx, int32_t M_new, int32_t first_new, float 
     WorkerRes fresh;
     if (e == cudaSuccess) {
         try {
-            e = make_worker_res(fresh, M_new, nt, ctx->nchunks, has_v, x, u, v);
+            e = make_worker_res(fresh, M_new, ctx->numel.data(), nt, ctx->total_elems, ctx->nrchunks, has_v, x, u, v);
             if (ctx->last_grads.capacity() < static_cast<size_t>(nptr_new))
                 ctx->last_grads.reserve(static_cast<size_t>(nptr_new));  // may throw; no state changed yet
         } catch (const std::bad_alloc &) {
@@ -651,7 +680,7 @@ int desloc_set_workers(desloc_ctx *ctx, int32_t M_new, int32_t first_new, float 
         const int n_arr = has_v ? 3 : 2;
         for (int arr = 0; arr < n_arr && e == cudaSuccess; ++arr)
             e = desloc::launch_mean_fill(
-                ctx->d_chunks, ctx->nchunks,
+                ctx->d_rchunks, ctx->nrchunks,
                 reinterpret_cast<const float *const *>(ctx->res.d_tables + arr * ctx->nptr), ctx->cfg.M,
                 reinterpret_cast<float *const *>(fresh.d_tables + arr * nptr_new +
                                                  static_cast<int64_t>(first_new) * nt),
@@ -705,6 +734,13 @@ int desloc_testing_set_max_blocks(desloc_ctx *ctx, int64_t max_blocks) {
     return DESLOC_OK;
 }
 
+int desloc_testing_set_wait_limit(desloc_ctx *ctx, int32_t polls) {
+    if (!ctx) return DESLOC_E_NULL;
+    ctx->wait_limit = polls < 0 ? desloc::DEFAULT_WAIT_LIMIT : polls;
+    if (polls < 0) *static_cast<volatile int *>(ctx->h_err) = 0;
+    return DESLOC_OK;
+}
+
 int desloc_last_cuda_error(const desloc_ctx *ctx) { return ctx ? ctx->last_cuda_error : 0; }
 
 const char *desloc_strerror(int status) {
@@ -716,6 +752,7 @@ const char *desloc_strerror(int status) {
         case DESLOC_E_NOMEM: return "out of memory";
         case DESLOC_E_CUDA: return "CUDA call failed";
         case DESLOC_E_TOO_LARGE: return "problem exceeds the fixed scratch of desloc_step_static";
+        case DESLOC_E_DEVICE_WAIT: return "a bounded wait on the device ran out in an earlier step";
         default: return "unknown status";
     }
 }

@@ -33,17 +33,15 @@ const void *lookup_sync(bool bf16, int mt, int mask) {
                 : pick_sync<OPT, POST, DIAG, float, FIRST, NMASK>(mt, mask, Seq{});
 }
 
-template <int OPT, bool DIAG>
-const void *lookup_local(bool bf16) {
-    return bf16 ? reinterpret_cast<const void *>(&desloc_local_kernel<OPT, bf16_t, DIAG>)
-                : reinterpret_cast<const void *>(&desloc_local_kernel<OPT, float, DIAG>);
-}
-
-// One unit per (optimizer, ordering, diagnostics): mt = 1 is the local kernel (pre units only).
+// One unit per (optimizer, ordering, diagnostics).  mt = 1 is the one-replica-per-tile kernel
+// (a single worker, or the local steps of more than MAX_MT workers); it lives in the pre units.
 template <int OPT, bool POST, bool DIAG>
 const void *lookup_unit(bool bf16, int mt, int mask) {
     if (mt == 1) {
-        if constexpr (!POST) return mask == 0 ? lookup_local<OPT, DIAG>(bf16) : nullptr;
+        if constexpr (!POST) {
+            if (mask != 0) return nullptr;
+            return bf16 ? kernel_ptr<OPT, false, DIAG, bf16_t, 1, 0>() : kernel_ptr<OPT, false, DIAG, float, 1, 0>();
+        }
         return nullptr;
     }
     return lookup_sync<OPT, POST, DIAG>(bf16, mt, mask);

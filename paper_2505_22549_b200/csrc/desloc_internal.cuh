@@ -13,6 +13,10 @@
 
 namespace desloc {
 
+// Polls a block gives its tile's copies before it gives up (each poll itself waits a while in
+// hardware): far beyond any healthy latency, still finite.
+constexpr int DEFAULT_WAIT_LIMIT = 1 << 22;
+
 // A named range around every step call, visible to tools that record NVTX (no cost otherwise).
 struct NvtxRange {
     explicit NvtxRange(const char *name) { nvtxRangePushA(name); }
@@ -75,12 +79,9 @@ inline uint32_t mask_at(const desloc_config *c, int64_t t) {
     return m;
 }
 
-// Chunk length for a tensor list.  Small problems (fewer full-size chunks than two per SM of a
-// B200) are latency-bound: quarter-size chunks spread them over four times as many blocks.
-inline int64_t chunk_elems_for(const int64_t *numel, int32_t num_tensors) {
-    int64_t full = 0;
-    for (int32_t k = 0; k < num_tensors; ++k) full += (numel[k] + CHUNK_ELEMS - 1) / CHUNK_ELEMS;
-    return full < 2 * 148 ? CHUNK_ELEMS / 4 : CHUNK_ELEMS;
+// Chunk length of a context with M workers: the tile of the kernel that serves it.
+inline int64_t chunk_elems_for(int32_t M) {
+    return M <= MAX_MT ? tile_elems(M) : GENERIC_CHUNK_ELEMS;
 }
 
 inline int64_t count_chunks(const int64_t *numel, int32_t num_tensors, int64_t chunk_elems) {
@@ -118,6 +119,8 @@ inline void fill_hyper(StepArgs &a, const desloc_config &c, float lr_t, float cl
     a.rho = c.clip_rho > 0.f ? c.clip_rho : std::numeric_limits<float>::infinity();
     a.cbound = (c.flags & DESLOC_FLAG_ADOPT_NORM_CLIP) ? clip_bound_t
                                                        : std::numeric_limits<float>::infinity();
+    a.wait_limit = DEFAULT_WAIT_LIMIT;
+    a.err = nullptr;
 }
 
 // Which kernel a step of this configuration runs, and over how many blocks.
@@ -138,7 +141,7 @@ inline LaunchPlan plan_launch(const desloc_config &c, uint32_t mask, long long n
     p.fn = generic ? lookup_generic_kernel(c.opt, post, bf16, static_cast<int>(kmask), diag)
                    : lookup_step_kernel(c.opt, post, bf16, c.M, static_cast<int>(kmask), diag);
     p.strides = !generic;
-    p.grid = per_worker_items ? ((nchunks + LOCAL_SLOTS - 1) / LOCAL_SLOTS) * c.M : nchunks;
+    p.grid = per_worker_items ? nchunks * c.M : nchunks;
     return p;
 }
 

@@ -109,7 +109,7 @@ sumsq_kernel(const Chunk *chunks, long long nchunks, const void *const *g, int n
                     const char *base =
                         reinterpret_cast<const char *>(g[static_cast<long long>(m) * nt + ch.tensor]) +
                         ch.start * static_cast<long long>(sizeof(GT));
-                    if (ch.count == CHUNK_ELEMS && (reinterpret_cast<uintptr_t>(base) & 15u) == 0)
+                    if (ch.count == REDUCE_CHUNK_ELEMS && (reinterpret_cast<uintptr_t>(base) & 15u) == 0)
                         wide[j] = reinterpret_cast<const uint4 *>(base);
                 }
             }

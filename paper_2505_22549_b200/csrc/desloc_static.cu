@@ -48,6 +48,7 @@ ScratchImage g_mirror;
 int g_mirror_device = -1;
 int32_t g_mirror_nt = 0;
 int64_t g_mirror_nptr = 0;
+int64_t g_mirror_chunk_elems = 0;
 int64_t g_mirror_numel[kMaxPointers];
 
 // First call on a device: resolve the device address of the scratch array with that device
@@ -85,7 +86,7 @@ extern "C" DESLOC_API int desloc_step_static(const desloc_config *cfg, float *co
     if (cfg->M > desloc::MAX_MT) return DESLOC_E_TOO_LARGE;
     const int64_t nptr = static_cast<int64_t>(cfg->M) * cfg->num_tensors;
     if (nptr > kMaxPointers) return DESLOC_E_TOO_LARGE;
-    const int64_t chunk_elems = desloc::chunk_elems_for(cfg->numel, cfg->num_tensors);
+    const int64_t chunk_elems = desloc::chunk_elems_for(cfg->M);
     const int64_t nchunks = desloc::count_chunks(cfg->numel, cfg->num_tensors, chunk_elems);
     if (nchunks > kMaxChunks) return DESLOC_E_TOO_LARGE;
     for (int64_t i = 0; i < nptr; ++i) {
@@ -121,6 +122,7 @@ extern "C" DESLOC_API int desloc_step_static(const desloc_config *cfg, float *co
         // What of the mirror still describes this device's array?
         const bool same_device = g_mirror_device == cuda_device;
         const bool same_plan = same_device && g_mirror_nt == cfg->num_tensors &&
+                               g_mirror_chunk_elems == chunk_elems &&
                                std::memcmp(g_mirror_numel, cfg->numel,
                                            static_cast<size_t>(cfg->num_tensors) * sizeof(int64_t)) == 0;
         const bool same_count = same_device && g_mirror_nptr == nptr;
@@ -133,6 +135,7 @@ extern "C" DESLOC_API int desloc_step_static(const desloc_config *cfg, float *co
             desloc::fill_chunks(cfg->numel, cfg->num_tensors, chunk_elems, g_mirror.chunks);
             std::memcpy(g_mirror_numel, cfg->numel, static_cast<size_t>(cfg->num_tensors) * sizeof(int64_t));
             g_mirror_nt = cfg->num_tensors;
+            g_mirror_chunk_elems = chunk_elems;
             e = cudaMemcpyAsync(base + offsetof(ScratchImage, chunks), g_mirror.chunks,
                                 static_cast<size_t>(nchunks) * sizeof(desloc::Chunk),
                                 cudaMemcpyHostToDevice, st);

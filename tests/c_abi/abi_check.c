@@ -30,9 +30,10 @@ int main(void) {
     CHECK(desloc_sync_mask(&cfg, 16) == (DESLOC_SYNC_X | DESLOC_SYNC_U));
     cfg.opt = DESLOC_ADAM;
 
-    CHECK(desloc_chunk_elems() == 4096);
+    CHECK(desloc_chunk_elems(4) == 512 && desloc_chunk_elems(1) == 1024 && desloc_chunk_elems(8) == 256);
+    CHECK(desloc_chunk_elems(0) == DESLOC_E_RANGE);
     int64_t out[3 * 8];
-    int64_t n = desloc_plan_chunks(numel, 3, desloc_chunk_elems(), out, 8);
+    int64_t n = desloc_plan_chunks(numel, 3, 4096, out, 8);
     CHECK(n == 5);
     CHECK(out[0] == 0 && out[1] == 0 && out[2] == 4096);
     CHECK(out[6] == 0 && out[7] == 8192 && out[8] == 10000 - 8192);

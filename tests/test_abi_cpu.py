@@ -62,8 +62,11 @@ def test_sync_mask_matches_oracle_schedule(d):
 
 
 def test_chunk_plan_covers_every_element_once(d):
-    ce = d.desloc_chunk_elems()
-    assert ce == 4096
+    assert [d.desloc_chunk_elems(M) for M in (1, 2, 3, 4, 5, 8, 9, 256)] == [1024, 1024, 512, 512, 256, 256, 1024, 1024]
+    for bad in (0, 257):
+        with pytest.raises(d.DeslocError):
+            d.desloc_chunk_elems(bad)
+    ce = 4096
     for numel in [[1], [ce], [ce + 1], [3, ce * 2, 5, ce * 3 - 1], list(di.mini(di.WORKLOADS["cfg2_adam_135m"]).numel)]:
         total, chunks = d.desloc_plan_chunks(numel, ce)
         assert total == len(chunks) == sum(-(-n // ce) for n in numel)
@@ -163,7 +166,8 @@ STATIC_BAD = [
     (dict(flags=8), "DESLOC_E_INVALID"), (dict(flags=1), "DESLOC_E_INVALID"),
     (dict(numel=[4, 0]), "DESLOC_E_RANGE"),
     (dict(numel=[1] * 1025), "DESLOC_E_TOO_LARGE"),                 # 2 x 1025 pointers
-    (dict(M=1, numel=[16384 * 4096 + 1]), "DESLOC_E_TOO_LARGE"),    # one chunk too many
+    (dict(M=1, numel=[32768 * 1024 + 1]), "DESLOC_E_TOO_LARGE"),    # one chunk too many
+    (dict(M=4, numel=[32768 * 512 + 1]), "DESLOC_E_TOO_LARGE"),
 ]
 
 

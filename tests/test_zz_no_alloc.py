@@ -62,7 +62,7 @@ def test_static_entry_point_rejects_what_does_not_fit():
     buf = torch.zeros(16, device=dev)
     p = buf.data_ptr()
     # too many chunks: one tensor of more than MAX_CHUNKS * chunk_elems parameters
-    big = d.DESLOC_STATIC_MAX_CHUNKS * d.desloc_chunk_elems() + 1
+    big = d.DESLOC_STATIC_MAX_CHUNKS * d.desloc_chunk_elems(1) + 1
     cfg = d.make_config(1, [big], "adam", "f32")
     with pytest.raises(d.DeslocError) as e:
         d.desloc_step_static(cfg, [p], [p], [p], [p], 0, 1e-3, 0.0, 0)
