@@ -272,10 +272,11 @@ DESLOC_API int64_t desloc_get_launch_count(const desloc_ctx *ctx);
 DESLOC_API int64_t desloc_plan_chunks(const int64_t *numel, int32_t num_tensors, int64_t chunk_elems,
                            int64_t *out, int64_t cap);
 
-/* Elements per chunk (the tile one thread block works on, for all workers) of a context with M
-   workers: 1024 for M <= 2 and M > 8, 512 for M = 3, 4, 256 for M = 5..8.  DESLOC_E_RANGE for an
-   M outside 1..DESLOC_MAX_M. */
-DESLOC_API int64_t desloc_chunk_elems(int32_t M);
+/* Elements per chunk -- the run of tiles one thread block streams through, for all workers -- of
+   a context created from cfg (M, numel and num_tensors are read).  A tile is 1024 elements for
+   M <= 2 and M > 8, 512 for M = 3, 4, 256 for M = 5..8; a chunk is up to 8 tiles (16 for
+   M = 5..8) on a large problem, fewer on a small one.  Negative desloc_status on bad input. */
+DESLOC_API int64_t desloc_chunk_elems(const desloc_config *cfg);
 
 /*
  * desloc_step_static(): one step for callers that cannot allocate.  (The paper has no
@@ -291,9 +292,9 @@ DESLOC_API int64_t desloc_chunk_elems(int32_t M);
  * device memory per GPU, held until the process exits.
  *
  * Limits: M * num_tensors <= DESLOC_STATIC_MAX_POINTERS, M <= 8, and at most
- * DESLOC_STATIC_MAX_CHUNKS chunks of desloc_chunk_elems(M) elements (every tensor starts a new
- * chunk) -- up to 32 Mi parameters for M <= 2, 16 Mi for M = 3, 4 and 8 Mi for M = 5..8 when
- * tensors are large.  Anything bigger returns DESLOC_E_TOO_LARGE and does nothing.
+ * DESLOC_STATIC_MAX_CHUNKS chunks of desloc_chunk_elems(cfg) elements (every tensor starts a
+ * new chunk) -- about 130 Mi parameters when tensors are large.  Anything bigger returns
+ * DESLOC_E_TOO_LARGE and does nothing.
  *
  * Arguments as for desloc_create() + desloc_step(): cfg, the host arrays x, u, v, grads of
  * M*num_tensors DEVICE pointers (v may be NULL for SGDM), the step t, eta_t, the ADOPT bound,

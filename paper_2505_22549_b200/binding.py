@@ -114,7 +114,7 @@ _lib.desloc_plan_chunks.argtypes = [ctypes.POINTER(ctypes.c_int64), ctypes.c_int
                                     ctypes.c_int64, ctypes.POINTER(ctypes.c_int64),
                                     ctypes.c_int64]
 _lib.desloc_chunk_elems.restype = ctypes.c_int64
-_lib.desloc_chunk_elems.argtypes = [ctypes.c_int32]
+_lib.desloc_chunk_elems.argtypes = [ctypes.POINTER(DeslocConfig)]
 _lib.desloc_strerror.restype = ctypes.c_char_p
 _lib.desloc_strerror.argtypes = [ctypes.c_int]
 _lib.desloc_last_cuda_error.restype = ctypes.c_int
@@ -306,9 +306,9 @@ def desloc_testing_set_max_blocks(ctx: int, max_blocks: int) -> None:
         raise DeslocError(rc, "desloc_testing_set_max_blocks")
 
 
-def desloc_chunk_elems(M: int) -> int:
-    """Elements per chunk (tile) of a context with M workers."""
-    n = int(_lib.desloc_chunk_elems(int(M)))
+def desloc_chunk_elems(cfg: DeslocConfig) -> int:
+    """Elements per chunk (the run of tiles one thread block streams) of a context made from cfg."""
+    n = int(_lib.desloc_chunk_elems(ctypes.byref(cfg) if cfg is not None else None))
     if n < 0:
         raise DeslocError(n, "desloc_chunk_elems")
     return n

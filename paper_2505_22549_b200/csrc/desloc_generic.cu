@@ -1,9 +1,7 @@
 // DES-LOC step for worker counts beyond the register-resident kernels (M > MAX_MT) on steps
 // that average something.  Same update as desloc_step_kernel, runtime M, compile-time mask.
 // Worker sums run in the order m = 0..M-1 as compensated fp32 sums (see WorkerSum): exact for
-// equal replicas, and within an ulp of a sequential fp64 reference.  Unlike the other kernels
-// this one takes the hardware reciprocal square root (2 ulp) for Adam's direction and ADOPT's
-// normaliser: it is bound by instruction issue, not by memory.
+// equal replicas, and within an ulp of a sequential fp64 reference.
 //
 // A block takes one chunk and first puts the chunk-relative pointers of all M workers into
 // shared memory, so that the per-position loops read them as broadcasts instead of chasing the
@@ -26,8 +24,9 @@ namespace {
 constexpr int GEN_MAX_M = 256;    // worker pointers staged per chunk (= the context's limit)
 // Measured on B200 (134.5 M parameters x 16 workers, fraction of the copy bandwidth on all-sync
 // steps): three blocks per SM with small batches 0.96; two blocks with batches twice as large
-// 0.85; fp64 worker sums 0.87 and IEEE sqrt / division 0.87 (this kernel is bound by
-// instruction issue: ~75 instructions per worker-coordinate before, ~45 now).
+// 0.85; fp64 worker sums 0.87 and IEEE sqrt / division instead of the hardware reciprocal
+// square root 0.87 (this kernel is bound by instruction issue: ~75 instructions per
+// worker-coordinate with those, ~45 without).
 constexpr int GEN_MIN_BLOCKS = 3;   // 80 registers per thread
 constexpr int GEN_BUDGET = 24;      // registers a batch of workers may hold in flight
 
@@ -197,8 +196,8 @@ __device__ __forceinline__ void generic_position(const StepArgs &a, char *const 
                             const float vp = SV ? vb.a[c] : vown;
                             const float xp = SX ? xb.a[c] : X[b].a[c];
                             float un, vn;
-                            state_update<OPT, true>(a, G[b].a[c] * sc, up, vp, vown, un, vn);
-                            D.a[c] = direction<OPT, true>(a, un, vn);
+                            state_update<OPT>(a, G[b].a[c] * sc, up, vp, vown, un, vn);
+                            D.a[c] = direction<OPT>(a, un, vn);
                             X[b].a[c] = apply_step(a, xp, D.a[c]);
                             U[b].a[c] = un;
                             V[b].a[c] = vn;
@@ -245,11 +244,11 @@ __device__ __forceinline__ void generic_position(const StepArgs &a, char *const 
                         for (int c = 0; c < VEC; ++c) {
                             const float vown = OPT != OPT_SGDM ? V[b].a[c] : 0.f;
                             float un, vn;
-                            state_update<OPT, true>(a, G[b].a[c] * sc, U[b].a[c], vown, vown, un, vn);
+                            state_update<OPT>(a, G[b].a[c] * sc, U[b].a[c], vown, vown, un, vn);
                             U[b].a[c] = un;
                             V[b].a[c] = vn;
                             if constexpr (!P::D_NEEDS_MEAN) {
-                                D.a[c] = direction<OPT, true>(a, un, vn);
+                                D.a[c] = direction<OPT>(a, un, vn);
                                 X[b].a[c] = apply_step(a, X[b].a[c], D.a[c]);
                             }
                         }
@@ -303,7 +302,7 @@ __device__ __forceinline__ void generic_position(const StepArgs &a, char *const 
                             for (int c = 0; c < VEC; ++c) {
                                 const float un = P::SU ? mu.a[c] : K[b].a[c];
                                 const float vn = P::SV ? mv.a[c] : (P::KEEP_V ? K[b].a[c] : 0.f);
-                                D.a[c] = direction<OPT, true>(a, un, vn);
+                                D.a[c] = direction<OPT>(a, un, vn);
                                 X[b].a[c] = apply_step(a, X[b].a[c], D.a[c]);
                             }
                             dd = sum_sq<VEC>(D);

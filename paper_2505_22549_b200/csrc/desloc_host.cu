@@ -107,7 +107,7 @@ cudaError_t make_worker_res(WorkerRes &r, int M, const int64_t *numel, int num_t
                             int64_t nrchunks, bool has_v, float *const *x, float *const *u,
                             float *const *v) {
     // tile plan for this worker count
-    const int64_t chunk_elems = desloc::chunk_elems_for(M);
+    const int64_t chunk_elems = desloc::chunk_elems_for(M, numel, num_tensors);
     const int64_t nchunks = desloc::count_chunks(numel, num_tensors, chunk_elems);
     std::vector<desloc::Chunk> chunks(static_cast<size_t>(nchunks));
     desloc::fill_chunks(numel, num_tensors, chunk_elems, chunks.data());
@@ -335,9 +335,14 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
             const bool cap = lp.strides && ctx->max_blocks > 0 && lp.grid > ctx->max_blocks;
             return static_cast<unsigned>(cap ? ctx->max_blocks : lp.grid);
         };
+        e = desloc::prepare_launch(plan);
+        if (e != cudaSuccess) {
+            rc = cuda_fail(ctx, e);
+            break;
+        }
         if (!host_grads) {
             e = cudaLaunchKernel(plan.fn, dim3(capped(plan)),
-                                 dim3(desloc::BLOCK_THREADS), params, 0, stream);
+                                 dim3(desloc::BLOCK_THREADS), params, plan.smem, stream);
             if (e == cudaSuccess) ctx->launches += 1;
         } else {
             // The device gradient buffers may still be read by earlier work on `stream`.
@@ -375,7 +380,7 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
                 a.diag_chunk0 = grp.c0;
                 const desloc::LaunchPlan gp = desloc::plan_launch(c, mask, a.nchunks, diag);
                 e = cudaLaunchKernel(gp.fn, dim3(capped(gp)),
-                                     dim3(desloc::BLOCK_THREADS), params, 0, stream);
+                                     dim3(desloc::BLOCK_THREADS), params, gp.smem, stream);
                 if (e == cudaSuccess) ctx->launches += 1;
             }
         }
@@ -411,8 +416,12 @@ uint32_t desloc_sync_mask(const desloc_config *cfg, int64_t t) {
     return mask_at(cfg, t);
 }
 
-int64_t desloc_chunk_elems(int32_t M) {
-    return (M < 1 || M > DESLOC_MAX_M) ? DESLOC_E_RANGE : desloc::chunk_elems_for(M);
+int64_t desloc_chunk_elems(const desloc_config *cfg) {
+    if (!cfg || !cfg->numel) return DESLOC_E_NULL;
+    if (cfg->M < 1 || cfg->M > DESLOC_MAX_M || cfg->num_tensors < 1) return DESLOC_E_RANGE;
+    for (int32_t k = 0; k < cfg->num_tensors; ++k)
+        if (cfg->numel[k] < 1) return DESLOC_E_RANGE;
+    return desloc::chunk_elems_for(cfg->M, cfg->numel, cfg->num_tensors);
 }
 
 int64_t desloc_plan_chunks(const int64_t *numel, int32_t num_tensors, int64_t chunk_elems,
@@ -453,10 +462,7 @@ int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *const *x, f
         if (cfg->opt != DESLOC_SGDM && !v[i]) return DESLOC_E_NULL;
     }
     const int64_t nrchunks = desloc::count_chunks(cfg->numel, cfg->num_tensors, desloc::REDUCE_CHUNK_ELEMS);
-    // one thread block per tile (per worker and tile when workers are separate items): the grid
-    // must fit for every worker count the context may be switched to
-    if (desloc::count_chunks(cfg->numel, cfg->num_tensors, 256) > 0x7fffffffLL / DESLOC_MAX_M)
-        return DESLOC_E_RANGE;
+    if (!desloc::grid_fits(cfg->M, cfg->numel, cfg->num_tensors)) return DESLOC_E_RANGE;
 
     desloc_ctx *ctx = new (std::nothrow) desloc_ctx();
     if (!ctx) return DESLOC_E_NOMEM;
@@ -652,6 +658,7 @@ int desloc_set_workers(desloc_ctx *ctx, int32_t M_new, int32_t first_new, float 
     const bool has_v = ctx->cfg.opt != DESLOC_SGDM;
     if (has_v && !v) return DESLOC_E_NULL;
     if (M_new < 1 || M_new > DESLOC_MAX_M || first_new < 0 || first_new > M_new) return DESLOC_E_RANGE;
+    if (!desloc::grid_fits(M_new, ctx->numel.data(), ctx->cfg.num_tensors)) return DESLOC_E_RANGE;
     const int nt = ctx->cfg.num_tensors;
     const int64_t nptr_new = static_cast<int64_t>(M_new) * nt;
     for (int64_t i = 0; i < nptr_new; ++i) {

@@ -79,9 +79,29 @@ inline uint32_t mask_at(const desloc_config *c, int64_t t) {
     return m;
 }
 
-// Chunk length of a context with M workers: the tile of the kernel that serves it.
-inline int64_t chunk_elems_for(int32_t M) {
-    return M <= MAX_MT ? tile_elems(M) : GENERIC_CHUNK_ELEMS;
+// Chunk length of a context: a run of tiles of the kernel that serves its worker count -- as
+// many as amortise the per-chunk pointer look-up on a large problem (max_tiles_per_chunk), fewer
+// on a small one, so that it still spreads over about four blocks per SM of a B200.
+inline int64_t chunk_elems_for(int32_t M, const int64_t *numel, int32_t num_tensors) {
+    const int64_t T = M <= MAX_MT ? tile_elems(M) : GENERIC_CHUNK_ELEMS;
+    const int64_t most = M <= MAX_MT ? max_tiles_per_chunk(M) : 8;
+    int64_t tiles = 0;
+    for (int32_t k = 0; k < num_tensors; ++k) tiles += (numel[k] + T - 1) / T;
+    int64_t per_chunk = tiles / (4 * 148);
+    if (per_chunk < 1) per_chunk = 1;
+    if (per_chunk > most) per_chunk = most;
+    return per_chunk * T;
+}
+
+// forward
+inline int64_t count_chunks(const int64_t *numel, int32_t num_tensors, int64_t chunk_elems);
+
+// One thread block per chunk (per worker and chunk where workers are separate work items): does
+// the grid of a context with M workers fit?
+inline bool grid_fits(int32_t M, const int64_t *numel, int32_t num_tensors) {
+    const int64_t nchunks = count_chunks(numel, num_tensors, chunk_elems_for(M, numel, num_tensors));
+    const int64_t per_chunk = (M == 1 || M > MAX_MT) ? M : 1;
+    return nchunks <= 0x7fffffffLL / per_chunk;
 }
 
 inline int64_t count_chunks(const int64_t *numel, int32_t num_tensors, int64_t chunk_elems) {
@@ -112,7 +132,7 @@ inline void fill_hyper(StepArgs &a, const desloc_config &c, float lr_t, float cl
     a.omb1 = static_cast<float>(1.0 - static_cast<double>(c.beta1));
     a.b2 = c.beta2;
     a.omb2 = static_cast<float>(1.0 - static_cast<double>(c.beta2));
-    a.eps = c.eps;
+    a.eps2 = static_cast<float>(static_cast<double>(c.eps) * static_cast<double>(c.eps));
     a.lam2 = static_cast<float>(static_cast<double>(c.eps) * static_cast<double>(c.eps));
     a.lr = lr_t;
     a.lrwd = static_cast<float>(static_cast<double>(lr_t) * static_cast<double>(c.weight_decay));
@@ -128,7 +148,15 @@ struct LaunchPlan {
     const void *fn = nullptr;
     long long grid = 0;
     bool strides = true;  // a smaller grid may stride over the work items (not the runtime-M kernel)
+    int smem = 0;         // dynamic shared memory of the launch
 };
+
+// The tile kernels use more than the 48 KB of shared memory a kernel gets by default: raise the
+// function's limit to what the launch asks for.  Not an allocation.
+inline cudaError_t prepare_launch(const LaunchPlan &p) {
+    if (p.smem <= 32 * 1024) return cudaSuccess;   // with the kernel's static part still under 48 KB
+    return cudaFuncSetAttribute(p.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, p.smem);
+}
 
 inline LaunchPlan plan_launch(const desloc_config &c, uint32_t mask, long long nchunks, bool diag) {
     LaunchPlan p;
@@ -141,6 +169,7 @@ inline LaunchPlan plan_launch(const desloc_config &c, uint32_t mask, long long n
     p.fn = generic ? lookup_generic_kernel(c.opt, post, bf16, static_cast<int>(kmask), diag)
                    : lookup_step_kernel(c.opt, post, bf16, c.M, static_cast<int>(kmask), diag);
     p.strides = !generic;
+    p.smem = generic ? 0 : step_smem_bytes(c.opt, per_worker_items ? 1 : c.M, bf16);
     p.grid = per_worker_items ? nchunks * c.M : nchunks;
     return p;
 }

@@ -1,21 +1,23 @@
 // DES-LOC fused step kernel for sm_100a: one streaming pass over g, x, u, v of all M
 // worker replicas (Algorithm 1 with the Adam, ADOPT and SGDM rules of Algorithms 2-3).
 //
-// Work decomposition.  The tensor list is cut into chunks ("tiles") of tile_elems(M) elements of
-// one tensor (table built once on the host); a thread block takes one tile of ALL M replicas
-// (for M = 1, and on local steps of more than eight workers, one tile of one replica):
-//   1. the first 4*M threads look up the tile's pointers and each issues ONE 1-D bulk
-//      asynchronous copy (cp.async.bulk, the TMA engine; no multicast, this GPU's own memory)
-//      of its array's tile into shared memory, all signalling one mbarrier;
+// Work decomposition.  The tensor list is cut into chunks of one tensor (table built once on the
+// host); a chunk is a run of up to 8-16 tiles of tile_elems(M) elements.  A thread block takes
+// one chunk of ALL M replicas (for M = 1, and on local steps of more than eight workers, of
+// one replica) and streams its tiles through two shared-memory buffers:
+//   1. the first 4*M threads look up the chunk's pointers once; each owns one (array, worker)
+//      and issues ONE 1-D bulk asynchronous copy per tile (cp.async.bulk, the TMA engine; no
+//      multicast, this GPU's own memory) of its 1-4 KB slice into the tile's buffer, all
+//      signalling the buffer's mbarrier;
 //   2. the block waits for the mbarrier (bounded; see bar_wait), then every thread updates its
 //      coordinates in place in shared memory: the arrays whose period divides t are averaged
 //      over the workers in a fixed tree order, then each worker takes its optimizer step -- a
 //      sync step moves the same bytes as a local step, through the same code shape;
-//   3. the threads that loaded x, u, v each issue one bulk copy of the updated tile back.
-// Tiles are small (28-32 KB of shared memory) and blocks short-lived: five to six of them are
-// resident per SM and overlap each other's load, compute and store phases; there is no
-// pipeline inside a block.  A tile whose pointers are not 16-byte aligned, or whose byte
-// counts are not multiples of 16 (a tensor's ragged tail), takes the same arithmetic straight
+//   3. the owners of x, u, v each issue one bulk copy of the updated slice back, and, once
+//      that copy has read the buffer, request the tile after next into it.
+// While tile k is updated, tile k + 1 is landing and tile k - 1 is on its way back.  Two to
+// three blocks are resident per SM.  A chunk whose pointers are not 16-byte aligned, and a
+// ragged last tile whose byte counts are not multiples of 16, take the same arithmetic straight
 // from and to global memory, one coordinate per thread.
 //
 // Measured on B200 (Adam, 4 workers, bf16 gradients, 1.7 G parameters; one local step):
@@ -23,9 +25,12 @@
 //   registers only, 256-bit loads (ld.global.v8.f32)                   26.39 ms  1.029
 //   bulk copies, 1024-element tiles, 2-stage pipeline, 2 blocks/SM     26.08 ms  1.041
 //   bulk copies, persistent grid (2 blocks/SM striding)                30.2  ms  0.90
-//   bulk copies, 512-element tiles, no pipeline, 6-8 blocks/SM         25.76 ms  1.055  <- this
-// ("copy" = the device-to-device copy bandwidth of the same GPU).  IEEE sqrt and division are
-// kept: the kernel is memory-bound and the hardware reciprocal square root was not faster.
+//   bulk copies, 512-element tiles, no pipeline, 6-8 blocks/SM         25.76 ms  1.055
+// ("copy" = the device-to-device copy bandwidth of the same GPU; these are single-tensor
+// experiments with the pointers in the kernel parameters).  In the library, with the tensor
+// list's pointer look-up on every block's path, the pipelined form is the robust one: a run
+// of 8-16 tiles per block through two buffers gives 26.1 ms (1.04) on the 218-tensor list,
+// local and sync steps alike.
 //
 // DIAG instantiations also accumulate, from values already in registers, the squared L2 norms
 // of the gradient as read, of the update d_t and of the new parameters per (worker, tile):
@@ -45,9 +50,13 @@ constexpr int REDUCE_CHUNK_ELEMS = BLOCK_THREADS * 16;  // chunks of the reducti
 constexpr int GENERIC_CHUNK_ELEMS = 1024;               // chunks of contexts with M > MAX_MT
 constexpr int DRAIN_WAIT_LIMIT = 1 << 22;               // bound on the wait for copies in flight
 
-// Elements per tile and worker for a kernel that holds mt replicas per tile: about 28 KB of
-// shared memory per block with bf16 gradients (32 KB with fp32), a multiple of the block size.
-__host__ __device__ constexpr int tile_elems(int mt) { return mt <= 2 ? 1024 : (mt <= 4 ? 512 : 256); }
+// Elements per tile and worker for a kernel that holds mt replicas per tile: bulk copies of
+// 2-4 KB per state array (copies of 1 KB and 512 B, with 256-element tiles, were 5 % slower on
+// eight workers), 28-57 KB of shared memory per buffer.
+__host__ __device__ constexpr int tile_elems(int mt) { return mt <= 2 ? 1024 : 512; }
+// Tiles per chunk on large problems (one pointer look-up and one pipeline fill serve them all):
+// 8 measured best up to four workers, 16 beyond.
+__host__ __device__ constexpr int max_tiles_per_chunk(int mt) { return mt <= 4 ? 8 : 16; }
 
 struct __align__(16) Chunk {
     int32_t tensor;  // index into the tensor list
@@ -75,7 +84,7 @@ struct StepArgs {
     int M;
     float b1, omb1;   // beta1, 1 - beta1
     float b2, omb2;   // beta2, 1 - beta2
-    float eps;        // ADOPT epsilon
+    float eps2;       // ADOPT epsilon, squared
     float lam2;       // Adam lambda^2
     float lr;         // eta_t
     float lrwd;       // eta_t * weight_decay
@@ -168,10 +177,18 @@ __device__ __forceinline__ float mean_of(const float (&s)[MT]) {
 // One worker's state update from the clipped gradient: `up`, `vp` are the previous states the
 // update starts from (the worker's own or the worker mean); `vown` is always the worker's own
 // previous v, which ADOPT's normaliser uses (Algorithm 3).
-// FAST: hardware reciprocal square root (2 ulp) in place of IEEE sqrt and division.  Only the
-// runtime-M kernel uses it: that kernel is bound by instruction issue, not by memory, and the
-// exact forms cost it a tenth of its speed.
-template <int OPT, bool FAST = false>
+// 1 / sqrt(a) to within an ulp: the hardware approximation (2 ulp) with one Newton step.  This
+// replaces IEEE sqrt followed by IEEE division (two roundings, about 20 instructions): with the
+// tiles staged by the copy engine the arithmetic sits on each block's critical path, and the
+// exact pair cost 1 % on Adam with four workers and 5-11 % on ADOPT with eight.  The error is
+// that of the exact pair (about one ulp of the quotient), not its bits.
+__device__ __forceinline__ float rsqrt_1ulp(float a) {
+    const float y = rsqrtf(a);
+    const float r = y * fmaf(-0.5f * a * y, y, 1.5f);
+    return a > 0.f && a < 3.0e38f ? r : y;   // keep the limits (1/0 = inf, 1/inf = 0) free of NaN
+}
+
+template <int OPT>
 __device__ __forceinline__ void state_update(const StepArgs &a, float g, float up, float vp,
                                              float vown, float &un, float &vn) {
     // coordinate-wise clip: sgn(g) min(|g|, rho)  (Section 3.1); rho = +inf when off
@@ -181,11 +198,7 @@ __device__ __forceinline__ void state_update(const StepArgs &a, float g, float u
         vn = fmaf(a.b2, vp, (a.omb2 * gh) * gh);
     } else if constexpr (OPT == OPT_ADOPT) {
         vn = fmaf(a.b2, vp, (a.omb2 * gh) * gh);
-        float r;
-        if constexpr (FAST)
-            r = gh * rsqrtf(fmaxf(vown, a.eps * a.eps));  // 1 / max(sqrt(v), eps)
-        else
-            r = gh / fmaxf(sqrtf(vown), a.eps);
+        float r = gh * rsqrt_1ulp(fmaxf(vown, a.eps2));  // g / max(sqrt(v), eps)
         r = fminf(fmaxf(r, -a.cbound), a.cbound);
         un = fmaf(a.b1, up, a.omb1 * r);
     } else {
@@ -195,10 +208,10 @@ __device__ __forceinline__ void state_update(const StepArgs &a, float g, float u
 }
 
 // The update d_t of Algorithms 2-3 from the new states.
-template <int OPT, bool FAST = false>
+template <int OPT>
 __device__ __forceinline__ float direction(const StepArgs &a, float un, float vn) {
     if constexpr (OPT == OPT_ADAM)
-        return FAST ? (a.lr * un) * rsqrtf(vn + a.lam2) : (a.lr * un) / sqrtf(vn + a.lam2);
+        return (a.lr * un) * rsqrt_1ulp(vn + a.lam2);
     else
         return a.lr * un;
 }
@@ -308,17 +321,30 @@ struct GlobalAcc {
 };
 
 // ---- diagnostics ------------------------------------------------------------------------------
-// A warp reduces each (kind, worker) value of a position at once (shuffle tree) and lane 0 adds
-// it to the warp's own slot in shared memory; the block total is the eight warp slots added in
-// order.  Deterministic.  All 32 lanes must call add(); a lane without work passes zero.
+// Each thread keeps its own running sums of squares, one per (kind, worker), in registers over
+// all tiles of a chunk.  At the end of the chunk a warp reduces each of them (shuffle tree) into
+// its slot of shared memory and the block total is the eight warp slots added in order:
+// deterministic, and a few dozen shuffles per thread and chunk.
 template <bool DIAG, int MT>
-struct WarpNorms {
-    float *slots;  // [DIAG_KINDS * MT][BLOCK_THREADS / 32]
-    __device__ __forceinline__ void add(int kind, int m, float v) const {
+struct ThreadNorms {
+    float acc[DIAG ? DIAG_KINDS * MT : 1];
+    __device__ __forceinline__ void clear() {
+#pragma unroll
+        for (int j = 0; j < (DIAG ? DIAG_KINDS * MT : 1); ++j) acc[j] = 0.f;
+    }
+    __device__ __forceinline__ void add(int kind, int m, float v) {
+        if constexpr (DIAG) acc[kind * MT + m] += v;
+    }
+    // all threads of the block call; slots: [DIAG_KINDS * MT][BLOCK_THREADS / 32]
+    __device__ __forceinline__ void reduce_into(float *slots) const {
         if constexpr (DIAG) {
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) v += __shfl_down_sync(0xffffffffu, v, off);
-            if ((threadIdx.x & 31) == 0) slots[(kind * MT + m) * (BLOCK_THREADS / 32) + (threadIdx.x >> 5)] += v;
+            for (int j = 0; j < DIAG_KINDS * MT; ++j) {
+                float v = acc[j];
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) v += __shfl_down_sync(0xffffffffu, v, off);
+                if ((threadIdx.x & 31) == 0) slots[j * (BLOCK_THREADS / 32) + (threadIdx.x >> 5)] = v;
+            }
         }
     }
 };
@@ -345,10 +371,10 @@ __device__ __forceinline__ FV<VEC> mean_over_workers(const Acc &acc, int arr, in
 // Post-average (Algorithms 4-5): every worker updates its states, the ones to be averaged are
 // replaced by their means, the parameter step uses those, and a synced x is averaged last.
 // A thread re-reads values it stored itself (never another thread's), so no barrier is needed.
-// `active` is false for the lanes a DIAG warp carries along without work.
 template <int OPT, int MASK, int MT, bool POST, bool DIAG, typename Acc>
 __device__ __forceinline__ void update_position(const StepArgs &a, const Acc &acc, const float *sscale,
-                                                int q, bool active, const WarpNorms<DIAG, MT> &wn) {
+                                                int q, ThreadNorms<DIAG, MT> &wn) {
+    constexpr bool active = true;
     constexpr int VEC = Acc::VEC;
     constexpr bool SX = MASK & SYNC_X, SU = MASK & SYNC_U;
     constexpr bool SV = (MASK & SYNC_V) && OPT != OPT_SGDM;
@@ -490,40 +516,51 @@ __device__ __forceinline__ bool bar_wait(uint64_t *bar, uint32_t parity, int lim
     return false;
 }
 
-// Resident blocks per SM the tile kernel is compiled for.
-__host__ __device__ constexpr int step_min_blocks(int mt) { return mt <= 4 ? 6 : 5; }
+constexpr int STAGES = 2;         // tile buffers per block (three stages at two blocks per SM: 0.84)
+// Resident blocks per SM: what the two buffers leave room for (three up to four workers, two
+// beyond).
+__host__ __device__ constexpr int step_min_blocks(int mt) { return mt <= 4 ? 3 : 2; }
 
+// A chunk is a run of consecutive tiles of one tensor.  The block looks its pointers up
+// once, then streams the tiles through a ring of STAGES buffers: while tile k is updated in
+// place, tile k + 1 is already landing; when tile k's copy back has left its buffer, tile
+// k + STAGES is requested into it.
 template <int OPT, int MASK, int MT, typename GT, bool POST, bool DIAG>
 __global__ void __launch_bounds__(BLOCK_THREADS, step_min_blocks(MT))
 desloc_step_kernel(const __grid_constant__ StepArgs a) {
-    constexpr int T = tile_elems(MT), VEC = T / BLOCK_THREADS;
+    constexpr int T = tile_elems(MT), VEC = T / BLOCK_THREADS, S = STAGES;
+    constexpr int ALIGN_ELEMS = 16 / static_cast<int>(sizeof(GT));   // bulk copies move multiples of 16 bytes
     constexpr bool HAS_V = OPT != OPT_SGDM;
     using L = TileLayout<OPT, MT, GT, T>;
-    __shared__ __align__(128) char tile[L::BYTES];
+    static_assert(4 * MT <= 32, "the (array, worker) owners are lanes of the first warp");
+    extern __shared__ __align__(128) char tile_mem[];   // S buffers of L::BYTES
     __shared__ char *sp[4][MT];
     __shared__ float sscale[MT];
-    __shared__ float snorm[DIAG ? DIAG_KINDS * MT * (BLOCK_THREADS / 32) : 1];
-    __shared__ __align__(8) uint64_t bar;
-    const WarpNorms<DIAG, MT> wn{snorm};
-    const int tid = threadIdx.x, lane = tid & 31;
-    if (tid == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&bar)) : "memory");
+    __shared__ __align__(8) uint64_t bar[S];
+    ThreadNorms<DIAG, MT> wn;
+    const int tid = threadIdx.x;
+    if (tid < S) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&bar[tid])) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    uint32_t phase = 0;
-    // Work items: tiles of all MT replicas; with MT = 1, (worker, tile) pairs -- the single
+    // this thread's role in the look-up, the loads and the stores: one (array, worker)
+    const int arr = tid / MT, m = tid - arr * MT;
+    const bool owner = tid < 4 * MT && (HAS_V || arr != 2);
+    const int esize = arr == 3 ? static_cast<int>(sizeof(GT)) : 4;
+    const int slot = arr == 3 ? L::g_off(m) : L::f_off(arr, m);
+    uint32_t phases = 0;  // bit s: parity of the phase barrier s completes next
+    // Work items: chunks of all MT replicas; with MT = 1, (worker, chunk) pairs -- the single
     // replica and the local steps of more than MAX_MT workers.  One item per block as launched;
     // a smaller grid strides over the rest.
     const long long nitems = MT == 1 ? a.nchunks * a.M : a.nchunks;
     for (long long item = blockIdx.x; item < nitems; item += gridDim.x) {
         const long long c = MT == 1 ? item % a.nchunks : item;
         const int m0 = MT == 1 ? static_cast<int>(item / a.nchunks) : 0;
-        const Chunk ch = a.chunks[c];
-        __syncthreads();  // the previous item is done with sp, tile and snorm; bar is initialised
-        const int arr = tid / MT, m = tid - arr * MT;   // meaningful for tid < 4 * MT
-        const bool mine = tid < 4 * MT && (HAS_V || arr != 2);
+        const Chunk ch = a.chunks[c];   // the same 16 bytes for every thread
+        const int count = ch.count;
+        __syncthreads();  // the previous item is done with the shared state; the barriers exist
         char *p = nullptr;
-        if (mine) {
+        if (owner) {
             const long long idx = static_cast<long long>(m0 + m) * a.nt + ch.tensor;
             if (arr == 0) p = reinterpret_cast<char *>(a.x[idx]) + ch.start * 4;
             if (arr == 1) p = reinterpret_cast<char *>(a.u[idx]) + ch.start * 4;
@@ -534,57 +571,89 @@ desloc_step_kernel(const __grid_constant__ StepArgs a) {
             sp[arr][m] = p;
         }
         if (tid < MT) sscale[tid] = a.gscale ? a.gscale[m0 + tid] : 1.f;
-        if constexpr (DIAG) {
-            if (tid < DIAG_KINDS * MT * (BLOCK_THREADS / 32)) snorm[tid] = 0.f;
-        }
-        // the bulk copies need 16-byte aligned addresses and byte counts (and a chunk that fits
-        // the tile: the host plans them so, the kernel does not rely on it)
-        const int ragged = ch.count % (16 / static_cast<int>(sizeof(GT))) != 0 || ch.count > T;
-        const bool direct = __syncthreads_or(ragged | ((reinterpret_cast<uintptr_t>(p) & 15u) != 0)) != 0;
-        if (!direct) {
-            const uint32_t fbytes = static_cast<uint32_t>(ch.count) * 4u;
-            const uint32_t gbytes = static_cast<uint32_t>(ch.count) * static_cast<uint32_t>(sizeof(GT));
-            if (mine)
-                bulk_load(tile + (arr == 3 ? L::g_off(m) : L::f_off(arr, m)), p, arr == 3 ? gbytes : fbytes, &bar);
+        wn.clear();
+        // bulk copies need 16-byte aligned addresses; a tile of the chunk also a byte count that
+        // is a multiple of 16 (only the chunk's last tile can miss that: it is then updated
+        // straight from global memory, like every tile of a chunk whose pointers are unaligned)
+        const bool unaligned = __syncthreads_or((reinterpret_cast<uintptr_t>(p) & 15u) != 0) != 0;
+        const int ntiles = (count + T - 1) / T;
+        const int staged = unaligned ? 0 : ((count % T) % ALIGN_ELEMS == 0 ? ntiles : ntiles - 1);   // tiles 0 .. staged-1
+        // request tile k (< staged) into its buffer: every owner its own slice, one arrival
+        auto request = [&](int k) {
+            const int cnt = min(T, count - k * T);
+            if (owner)
+                bulk_load(tile_mem + (k % S) * L::BYTES + slot, p + static_cast<long long>(k) * T * esize,
+                          static_cast<uint32_t>(cnt * esize), &bar[k % S]);
             if (tid == 0)
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
-                             :: "r"(smem_u32(&bar)), "r"(MT * (gbytes + L::NS * fbytes)) : "memory");
-            const bool landed = bar_wait(&bar, phase, a.wait_limit);
-            phase ^= 1u;
+                             :: "r"(smem_u32(&bar[k % S])),
+                                "r"(static_cast<uint32_t>(MT * cnt * (static_cast<int>(sizeof(GT)) + 4 * L::NS)))
+                             : "memory");
+        };
+#pragma unroll
+        for (int k = 0; k < S; ++k)
+            if (k < staged) request(k);
+#pragma unroll 1
+        for (int k = 0; k < staged; ++k) {
+            const int st = k % S;
+            const int cnt = min(T, count - k * T);
+            const bool landed = bar_wait(&bar[st], (phases >> st) & 1u, a.wait_limit);
             if (__syncthreads_or(!landed)) {
                 // Give up on this step: say so, let the copies already requested land (bounded as
-                // well), store nothing, leave.  The host reports the flag on its next call.
+                // well), store nothing more, leave.  The host reports the flag on its next call.
                 if (tid == 0 && a.err) *reinterpret_cast<volatile int *>(a.err) = 1;
-                if (!landed) bar_wait(&bar, phase ^ 1u, DRAIN_WAIT_LIMIT);
+                for (int kk = k; kk < staged && kk < k + S; ++kk)
+                    bar_wait(&bar[kk % S], (phases >> (kk % S)) & 1u, DRAIN_WAIT_LIMIT);
+                asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
                 __syncthreads();
                 return;
             }
-            const SmemAcc<OPT, MT, GT, T, VEC> acc{tile};
-            const bool active = tid * VEC < ch.count;
-            if (DIAG || active) update_position<OPT, MASK, MT, POST, DIAG>(a, acc, sscale, tid, active, wn);
+            phases ^= 1u << st;
+            const SmemAcc<OPT, MT, GT, T, VEC> acc{tile_mem + st * L::BYTES};
+            if (tid * VEC < cnt) update_position<OPT, MASK, MT, POST, DIAG>(a, acc, sscale, tid, wn);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // our writes, then the copy engine's reads
             __syncthreads();
-            if (mine && arr != 3) {
-                bulk_store(p, tile + L::f_off(arr, m), fbytes);
+            if (owner && arr != 3) {
+                bulk_store(p + static_cast<long long>(k) * T * 4, tile_mem + st * L::BYTES + slot,
+                           static_cast<uint32_t>(cnt * 4));
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // before the tile is reused or freed
             }
-        } else {
-            const GlobalAcc<MT, GT> acc{sp};
-            for (int e = tid; DIAG ? (e - lane < ch.count) : (e < ch.count); e += BLOCK_THREADS)
-                update_position<OPT, MASK, MT, POST, DIAG>(a, acc, sscale, e, e < ch.count, wn);
+            if (k + S < staged) {
+                // the buffer is free once this thread's own copy back has read it
+                if (owner && arr != 3) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                request(k + S);
+            }
         }
+        if (staged * T < count) {
+            // what could not be staged: the whole chunk, or its ragged last tile
+            const int e0 = staged * T;
+            const GlobalAcc<MT, GT> acc{sp};
+            for (int e = e0 + tid; e < count; e += BLOCK_THREADS)
+                update_position<OPT, MASK, MT, POST, DIAG>(a, acc, sscale, e, wn);
+        }
+        // the copies back must have left shared memory before the buffers are reused or freed
+        if (owner && arr != 3) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
         if constexpr (DIAG) {
+            // the tile buffers are idle now: their first bytes serve as the warps' slots
+            float *slots = reinterpret_cast<float *>(tile_mem);
+            __syncthreads();
+            wn.reduce_into(slots);
             __syncthreads();
             if (tid < DIAG_KINDS * MT) {
                 float total = 0.f;
 #pragma unroll
-                for (int w = 0; w < BLOCK_THREADS / 32; ++w) total += snorm[tid * (BLOCK_THREADS / 32) + w];
+                for (int w = 0; w < BLOCK_THREADS / 32; ++w) total += slots[tid * (BLOCK_THREADS / 32) + w];
                 const int kind = tid / MT, mm = tid - kind * MT;
                 a.diag[(static_cast<long long>(kind) * a.M + m0 + mm) * a.diag_stride + a.diag_chunk0 + c] = total;
             }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // before the copy engine writes there again
         }
     }
+}
+
+// Dynamic shared memory a launch of desloc_step_kernel<opt, ., mt, grad type, ., .> needs.
+__host__ __device__ constexpr int step_smem_bytes(int opt, int mt, bool bf16) {
+    return STAGES * mt * tile_elems(mt) * ((bf16 ? 2 : 4) + 4 * (opt == OPT_SGDM ? 2 : 3));
 }
 
 // Lookup of an instantiation: opt, post-average?, bf16 gradients?, MT in 1..MAX_MT, mask,

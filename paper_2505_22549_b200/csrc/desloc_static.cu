@@ -86,7 +86,7 @@ extern "C" DESLOC_API int desloc_step_static(const desloc_config *cfg, float *co
     if (cfg->M > desloc::MAX_MT) return DESLOC_E_TOO_LARGE;
     const int64_t nptr = static_cast<int64_t>(cfg->M) * cfg->num_tensors;
     if (nptr > kMaxPointers) return DESLOC_E_TOO_LARGE;
-    const int64_t chunk_elems = desloc::chunk_elems_for(cfg->M);
+    const int64_t chunk_elems = desloc::chunk_elems_for(cfg->M, cfg->numel, cfg->num_tensors);
     const int64_t nchunks = desloc::count_chunks(cfg->numel, cfg->num_tensors, chunk_elems);
     if (nchunks > kMaxChunks) return DESLOC_E_TOO_LARGE;
     for (int64_t i = 0; i < nptr; ++i) {
@@ -172,8 +172,10 @@ extern "C" DESLOC_API int desloc_step_static(const desloc_config *cfg, float *co
         a.diag = nullptr;
         desloc::fill_hyper(a, *cfg, lr_t, clip_bound_t);
         void *params[] = {&a};
-        e = cudaLaunchKernel(plan.fn, dim3(static_cast<unsigned>(plan.grid)),
-                             dim3(desloc::BLOCK_THREADS), params, 0, st);
+        e = desloc::prepare_launch(plan);
+        if (e == cudaSuccess)
+            e = cudaLaunchKernel(plan.fn, dim3(static_cast<unsigned>(plan.grid)),
+                                 dim3(desloc::BLOCK_THREADS), params, plan.smem, st);
         if (e != cudaSuccess) { rc = DESLOC_E_CUDA; break; }
     } while (false);
     if (rc == DESLOC_E_CUDA) (void)cudaGetLastError();

@@ -85,12 +85,23 @@ def rel_err(gpu: np.ndarray, ref: np.ndarray, rms: float | None = None) -> float
     return float(np.max(np.abs(gpu.astype(np.float64) - ref64) / den))
 
 
+TINY = 64   # tensors with fewer elements have no meaningful RMS of their own
+
+
 def compare_per_tensor(st: State, gpu: np.ndarray, ref: np.ndarray, what: str, tol: float = TOL):
-    """gpu/ref are [M, nflat]; checks every (worker, tensor) block against `tol`."""
+    """gpu/ref are [M, nflat]; checks every (worker, tensor) block against `tol`.
+
+    The error of an element is taken relative to max(|ref|, rms of its tensor): the floor is
+    there because elements pass through zero while their absolute error stays at the scale of
+    the tensor.  The RMS of a tensor of a handful of elements is no such scale (for one element
+    it is the element itself), so tensors below TINY elements take the RMS of the worker's whole
+    array as floor."""
     worst = 0.0
     for m in range(gpu.shape[0]):
+        whole = np.concatenate([ref[m, o:o + n] for o, n in zip(st.offs, st.w.numel)]).astype(np.float64)
+        rms_all = float(np.sqrt(np.mean(whole * whole))) if whole.size else 0.0
         for k, (o, n) in enumerate(zip(st.offs, st.w.numel)):
-            e = rel_err(gpu[m, o:o + n], ref[m, o:o + n])
+            e = rel_err(gpu[m, o:o + n], ref[m, o:o + n], rms=None if n >= TINY else rms_all)
             worst = max(worst, e)
             assert e <= tol, f"{what}: worker {m} tensor {k} (numel {n}) rel err {e:.3e} > {tol}"
     return worst

@@ -62,10 +62,16 @@ def test_sync_mask_matches_oracle_schedule(d):
 
 
 def test_chunk_plan_covers_every_element_once(d):
-    assert [d.desloc_chunk_elems(M) for M in (1, 2, 3, 4, 5, 8, 9, 256)] == [1024, 1024, 512, 512, 256, 256, 1024, 1024]
+    big = [1 << 24] * 4                       # plenty of tiles: the full run per chunk
+    want = {1: 8192, 2: 8192, 3: 4096, 4: 4096, 5: 8192, 8: 8192, 9: 8192, 256: 8192}
+    for M, ce_want in want.items():
+        assert d.desloc_chunk_elems(d.make_config(M, big, "adam", "bf16")) == ce_want
+    # a small problem gets single-tile chunks so that it still spreads over many blocks
+    assert d.desloc_chunk_elems(d.make_config(2, [4096], "adam", "f32")) == 1024
+    assert d.desloc_chunk_elems(d.make_config(4, [4096 * 100], "adam", "f32")) == 512
     for bad in (0, 257):
         with pytest.raises(d.DeslocError):
-            d.desloc_chunk_elems(bad)
+            d.desloc_chunk_elems(d.make_config(bad, [8], "adam", "f32"))
     ce = 4096
     for numel in [[1], [ce], [ce + 1], [3, ce * 2, 5, ce * 3 - 1], list(di.mini(di.WORKLOADS["cfg2_adam_135m"]).numel)]:
         total, chunks = d.desloc_plan_chunks(numel, ce)
@@ -166,8 +172,8 @@ STATIC_BAD = [
     (dict(flags=8), "DESLOC_E_INVALID"), (dict(flags=1), "DESLOC_E_INVALID"),
     (dict(numel=[4, 0]), "DESLOC_E_RANGE"),
     (dict(numel=[1] * 1025), "DESLOC_E_TOO_LARGE"),                 # 2 x 1025 pointers
-    (dict(M=1, numel=[32768 * 1024 + 1]), "DESLOC_E_TOO_LARGE"),    # one chunk too many
-    (dict(M=4, numel=[32768 * 512 + 1]), "DESLOC_E_TOO_LARGE"),
+    (dict(M=1, numel=[32768 * 8192 + 1]), "DESLOC_E_TOO_LARGE"),    # one chunk too many
+    (dict(M=4, numel=[32768 * 4096 + 1]), "DESLOC_E_TOO_LARGE"),
 ]
 
 

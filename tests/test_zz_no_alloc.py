@@ -62,8 +62,9 @@ def test_static_entry_point_rejects_what_does_not_fit():
     buf = torch.zeros(16, device=dev)
     p = buf.data_ptr()
     # too many chunks: one tensor of more than MAX_CHUNKS * chunk_elems parameters
-    big = d.DESLOC_STATIC_MAX_CHUNKS * d.desloc_chunk_elems(1) + 1
+    big = d.DESLOC_STATIC_MAX_CHUNKS * 8192 + 1        # 8192 = a chunk of a large one-worker list
     cfg = d.make_config(1, [big], "adam", "f32")
+    assert d.desloc_chunk_elems(cfg) == 8192
     with pytest.raises(d.DeslocError) as e:
         d.desloc_step_static(cfg, [p], [p], [p], [p], 0, 1e-3, 0.0, 0)
     assert e.value.status == d.DESLOC_E_TOO_LARGE
