@@ -516,7 +516,7 @@ def run_ours(args, w):
 # the ncu captures summarised under profiles/ (44 M-parameter stand-ins of the workloads: the
 # full sizes are too large for a multi-pass capture; each byte is touched once, so traffic grows
 # in proportion to the parameter count).  Keyed by (optimizer, M).
-TRAFFIC_PER_ALGORITHMIC_BYTE = {("adam", 4): 0.9876, ("adopt", 8): 0.9938}
+TRAFFIC_PER_ALGORITHMIC_BYTE = {("adam", 4): 0.9875, ("adopt", 8): 0.9937}
 
 
 def run_e2e(args, w, eng, G, X, offs, dev, world, barrier):

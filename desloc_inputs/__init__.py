@@ -106,6 +106,11 @@ def _wl() -> dict:
                                                         K=(4, 8, 16), T=16)
     w["prof_adopt_m8_44m"] = w["cfg3_adopt_360m"].replace(name="prof_adopt_m8_44m", numel=prof,
                                                           K=(4, 8, 16), T=16)
+    # Sixteen workers (the runtime-M kernel on sync steps) on a 3-block model: 25 M parameters,
+    # 5.7 GB resident; every step syncs all three arrays.
+    w["prof_adam_m16_25m"] = w["cfg2_adam_135m"].replace(
+        name="prof_adam_m16_25m", M=16, numel=tuple(llama_tensor_list(3, 768, 256, 2048, 8192)),
+        K=(1, 1, 1), T=16)
     return w
 
 
