@@ -200,7 +200,7 @@ DESLOC_API int desloc_get_grad_norms(desloc_ctx *ctx, float *norms_out, float *s
  *           eta_t u_t for ADOPT and SGDM; the weight-decay term is not part of it)
  * -- the gradient, parameter and update norms the paper tracks (gradient norms after the
  * workers are doubled, Section 6, RQ3; update and parameter norms of the billion-scale runs,
- * additional-results appendix).  The step kernel already holds all three in registers, so the
+ * additional-results appendix).  The step kernel already has all three on chip, so the
  * sums of squares are formed there, one partial per (kind, worker, chunk): no extra pass over
  * memory, and the step computes exactly what desloc_step() computes.
  *   max_norm : > 0 puts norm-based clipping in front as desloc_step_normclip() does; 0 = off.

@@ -33,8 +33,8 @@
 // local and sync steps alike.
 //
 // DIAG instantiations also accumulate, from values already in registers, the squared L2 norms
-// of the gradient as read, of the update d_t and of the new parameters per (worker, tile):
-// no extra pass over memory, 12 bytes written per worker and tile.
+// of the gradient as read, of the update d_t and of the new parameters per (worker, chunk):
+// no extra pass over memory, 12 bytes written per worker and chunk.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
