@@ -20,15 +20,40 @@ CASES = [
     ("cfg2_adam_135m", 40, 0, 1 << 17),
     ("cfg3_adopt_360m", 20, 0, 1 << 16),
     ("cfg4_adam_1p7b", 24, 56, 1 << 17),     # t = 56..79 crosses the x-sync at t = 64
+    # workload 5: both optimizers under its three schedules (every step / every 16 / 16-64-256)
+    ("cfg5_sgdm_ddp", 4, 0, 1 << 16),
+    ("cfg5_sgdm_local", 18, 0, 1 << 16),
     ("cfg5_sgdm_desloc", 18, 0, 1 << 16),
     ("cfg5_adam_ddp", 6, 0, 1 << 16),
+    ("cfg5_adam_local", 18, 0, 1 << 16),
+    ("cfg5_adam_desloc", 18, 0, 1 << 16),
+]
+
+# The other orderings and kernels at full size: (workload, workers or None, post-average, steps)
+VARIANTS = [
+    ("cfg3_adopt_360m", None, True, 12),     # Algorithm 4-5 ordering, eight workers
+    ("cfg2_adam_135m", None, True, 12),
+    ("cfg2_adam_135m", 16, False, 12),       # more than eight workers: runtime-M kernel on sync steps
+    ("cfg2_adam_135m", 16, True, 6),
+    ("cfg5_sgdm_desloc", 3, False, 18),      # a worker count that is not a power of two
 ]
 
 
 @pytest.mark.parametrize("name,T,t0,nsamp", CASES)
 def test_fullsize_sampled_parity(name, T, t0, nsamp):
-    import paper_2505_22549_b200 as d
+    _sampled_parity(di.WORKLOADS[name], name, T, t0, nsamp, post=False)
+
+
+@pytest.mark.parametrize("name,M,post,T", VARIANTS)
+def test_fullsize_sampled_parity_of_other_orderings_and_worker_counts(name, M, post, T):
     w = di.WORKLOADS[name]
+    if M is not None:
+        w = w.replace(M=M, K=(4, 8, 12))     # sync steps of every kind within a short run
+    _sampled_parity(w, f"{name} M={w.M} post={post}", T, 0, 1 << 15, post=post)
+
+
+def _sampled_parity(w, name, T, t0, nsamp, post):
+    import paper_2505_22549_b200 as d
     dev = torch.device("cuda:0")
     free, _ = torch.cuda.mem_get_info()
     need = w.N * w.M * (14 if w.opt != "sgdm" else 10) + (6 << 30)
@@ -41,12 +66,12 @@ def test_fullsize_sampled_parity(name, T, t0, nsamp):
             di.fill_grads_(w, 10_000 + m, m, st.g[m], align=4)
             st.u[m].copy_(st.g[m])
             st.v[m].copy_(st.g[m]).square_()
-    eng = make_engine(d, w, st)
+    eng = make_engine(d, w, st, post)
     idx_np = di.sample_indices(w.numel, nsamp, seed=1, align=4)
     idx = torch.from_numpy(idx_np).to(dev)
     ox, ou = st.to_numpy(st.x, idx), st.to_numpy(st.u, idx)
     ov = st.to_numpy(st.v, idx) if st.v is not None else None
-    ocfg = oracle_cfg(w)
+    ocfg = oracle_cfg(w, oracle.FLAG_POST_AVERAGE if post else 0)
     gviews = st.views(st.g)
     for t in range(t0, t0 + T):
         st.fill_grads(t)
