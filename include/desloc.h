@@ -216,7 +216,8 @@ DESLOC_API int desloc_step_diag(desloc_ctx *ctx, int64_t t, float lr_t, float cl
  *                    or NULL;
  *   total_out      : host, [3][M] floats, the norm over the whole tensor list, or NULL.
  * Per-chunk partials are fp32; they are added per tensor, and the tensors per worker, in fp64
- * in a fixed order (deterministic, no atomics).  Two small launches on `stream`, then the
+ * in a fixed order (no atomics: the same buffers and inputs give the same bits; where the chunks
+ * of a tensor begin follows the alignment of worker 0's x, see desloc_plan_chunks_at()).  Two small launches on `stream`, then the
  * copies; the call waits for `stream`.  DESLOC_E_INVALID if no diagnostics step has run since
  * the context was created or its workers were changed.
  */
@@ -263,19 +264,29 @@ DESLOC_API int desloc_get_counters(const desloc_ctx *ctx, int64_t out[4]);
 DESLOC_API int64_t desloc_get_launch_count(const desloc_ctx *ctx);
 
 /*
- * Multi-tensor plan: how the tensor list is cut into the fixed-size chunks that thread
- * blocks work through.  Host-only.  Writes up to `cap` chunks as triples
- * (tensor index, first element, element count) into `out` (3*cap int64) and returns the total
- * number of chunks the list needs (which may exceed cap), or a negative desloc_status.
- * Every tensor starts a new chunk; chunks of a tensor are `chunk_elems` long except the last.
+ * Multi-tensor plan: how the tensor list is cut into the chunks that thread blocks work
+ * through.  Host-only.  Writes up to `cap` chunks as triples (tensor index, first element,
+ * element count) into `out` (3*cap int64) and returns the total number of chunks the list
+ * needs (which may exceed cap), or a negative desloc_status.
+ * Every tensor starts a new chunk; chunks of a tensor are `chunk_elems` long except the last --
+ * and except the first, where x0 says so:
+ *   x0 : host array of num_tensors addresses, worker 0's x tensors (never dereferenced), or NULL.
+ *        The copy engine is fastest on pieces that start on a 2 KB boundary, so when the address
+ *        of a tensor is a multiple of 32 bytes but not of 2 KB, its first chunk is cut to the
+ *        elements in front of the next 2 KB boundary and every later chunk starts on one.
+ * desloc_plan_chunks_at() with the x pointers given to desloc_create() is the table that context
+ * works from; desloc_plan_chunks() is the same with x0 = NULL.
  */
+DESLOC_API int64_t desloc_plan_chunks_at(const int64_t *numel, int32_t num_tensors, int64_t chunk_elems,
+                                         const void *const *x0, int64_t *out, int64_t cap);
 DESLOC_API int64_t desloc_plan_chunks(const int64_t *numel, int32_t num_tensors, int64_t chunk_elems,
-                           int64_t *out, int64_t cap);
+                                      int64_t *out, int64_t cap);
 
 /* Elements per chunk -- the run of tiles one thread block streams through, for all workers -- of
    a context created from cfg (M, numel and num_tensors are read).  A tile is 1024 elements for
-   M <= 2 and M > 8, 512 for M = 3, 4, 256 for M = 5..8; a chunk is up to 8 tiles (16 for
-   M = 5..8) on a large problem, fewer on a small one.  Negative desloc_status on bad input. */
+   M <= 2, 512 for M = 3..8 (M > 8: 1024-element chunks, no tiles); a chunk is up to 8 tiles
+   on a large problem, fewer on a small one.  Negative desloc_status on bad
+   input. */
 DESLOC_API int64_t desloc_chunk_elems(const desloc_config *cfg);
 
 /*

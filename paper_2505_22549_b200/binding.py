@@ -113,6 +113,10 @@ _lib.desloc_plan_chunks.restype = ctypes.c_int64
 _lib.desloc_plan_chunks.argtypes = [ctypes.POINTER(ctypes.c_int64), ctypes.c_int32,
                                     ctypes.c_int64, ctypes.POINTER(ctypes.c_int64),
                                     ctypes.c_int64]
+_lib.desloc_plan_chunks_at.restype = ctypes.c_int64
+_lib.desloc_plan_chunks_at.argtypes = [ctypes.POINTER(ctypes.c_int64), ctypes.c_int32,
+                                       ctypes.c_int64, ctypes.POINTER(ctypes.c_void_p),
+                                       ctypes.POINTER(ctypes.c_int64), ctypes.c_int64]
 _lib.desloc_chunk_elems.restype = ctypes.c_int64
 _lib.desloc_chunk_elems.argtypes = [ctypes.POINTER(DeslocConfig)]
 _lib.desloc_strerror.restype = ctypes.c_char_p
@@ -322,15 +326,25 @@ def desloc_testing_set_wait_limit(ctx: int, polls: int) -> None:
         raise DeslocError(rc, "desloc_testing_set_wait_limit")
 
 
-def desloc_plan_chunks(numel: Sequence[int], chunk_elems: int, cap: Optional[int] = None):
-    """Returns (total_chunks, [(tensor, start, count), ...] up to cap)."""
+def desloc_plan_chunks(numel: Sequence[int], chunk_elems: int, cap: Optional[int] = None,
+                       x0: Optional[Sequence[int]] = None):
+    """Returns (total_chunks, [(tensor, start, count), ...] up to cap).  x0: the addresses of
+    worker 0's x tensors (desloc_plan_chunks_at: first chunks cut at 2 KB boundaries) or None."""
     arr = (ctypes.c_int64 * max(1, len(numel)))(*[int(n) for n in numel])
-    total = _lib.desloc_plan_chunks(arr, len(numel), int(chunk_elems), None, 0)
+    xs = None
+    if x0 is not None:
+        if len(x0) != len(numel):
+            raise ValueError("x0 must hold one address per tensor")
+        xs = (ctypes.c_void_p * max(1, len(x0)))(*[int(p) for p in x0])
+    total = _lib.desloc_plan_chunks_at(arr, len(numel), int(chunk_elems), xs, None, 0)
     if total < 0:
         raise DeslocError(int(total), "desloc_plan_chunks")
     cap = total if cap is None else min(cap, total)
     out = (ctypes.c_int64 * max(1, 3 * cap))()
-    total2 = _lib.desloc_plan_chunks(arr, len(numel), int(chunk_elems), out, cap)
+    if x0 is None:
+        total2 = _lib.desloc_plan_chunks(arr, len(numel), int(chunk_elems), out, cap)
+    else:
+        total2 = _lib.desloc_plan_chunks_at(arr, len(numel), int(chunk_elems), xs, out, cap)
     assert total2 == total
     return int(total), [(int(out[3 * i]), int(out[3 * i + 1]), int(out[3 * i + 2]))
                         for i in range(cap)]

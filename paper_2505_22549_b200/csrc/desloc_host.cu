@@ -108,9 +108,11 @@ cudaError_t make_worker_res(WorkerRes &r, int M, const int64_t *numel, int num_t
                             float *const *v) {
     // tile plan for this worker count
     const int64_t chunk_elems = desloc::chunk_elems_for(M, numel, num_tensors);
-    const int64_t nchunks = desloc::count_chunks(numel, num_tensors, chunk_elems);
+    std::vector<int64_t> heads(static_cast<size_t>(num_tensors));
+    for (int32_t k = 0; k < num_tensors; ++k) heads[k] = desloc::head_elems(x[k], numel[k]);
+    const int64_t nchunks = desloc::count_chunks(numel, num_tensors, chunk_elems, heads.data());
     std::vector<desloc::Chunk> chunks(static_cast<size_t>(nchunks));
-    desloc::fill_chunks(numel, num_tensors, chunk_elems, chunks.data());
+    desloc::fill_chunks(numel, num_tensors, chunk_elems, chunks.data(), heads.data());
     std::vector<long long> tstart(static_cast<size_t>(num_tensors) + 1, 0);
     r.groups.clear();
     {
@@ -118,7 +120,7 @@ cudaError_t make_worker_res(WorkerRes &r, int M, const int64_t *numel, int num_t
         int64_t acc = 0, c0 = 0;
         int32_t k0 = 0;
         for (int32_t k = 0; k < num_tensors; ++k) {
-            tstart[k + 1] = tstart[k] + (numel[k] + chunk_elems - 1) / chunk_elems;
+            tstart[k + 1] = tstart[k] + desloc::chunks_of(numel[k], chunk_elems, heads[k]);
             acc += numel[k];
             const int done_groups = static_cast<int>(r.groups.size());
             const bool last = k == num_tensors - 1;
@@ -424,24 +426,37 @@ int64_t desloc_chunk_elems(const desloc_config *cfg) {
     return desloc::chunk_elems_for(cfg->M, cfg->numel, cfg->num_tensors);
 }
 
-int64_t desloc_plan_chunks(const int64_t *numel, int32_t num_tensors, int64_t chunk_elems,
-                           int64_t *out, int64_t cap) {
+int64_t desloc_plan_chunks_at(const int64_t *numel, int32_t num_tensors, int64_t chunk_elems,
+                              const void *const *x0, int64_t *out, int64_t cap) {
     if (!numel) return DESLOC_E_NULL;
     if (num_tensors < 1 || chunk_elems < 1 || cap < 0) return DESLOC_E_RANGE;
     if (cap > 0 && !out) return DESLOC_E_NULL;
-    int64_t n = 0;
-    for (int32_t k = 0; k < num_tensors; ++k) {
+    for (int32_t k = 0; k < num_tensors; ++k)
         if (numel[k] < 1) return DESLOC_E_RANGE;
-        for (int64_t s = 0; s < numel[k]; s += chunk_elems) {
-            if (n < cap) {
-                out[3 * n + 0] = k;
-                out[3 * n + 1] = s;
-                out[3 * n + 2] = (numel[k] - s < chunk_elems) ? numel[k] - s : chunk_elems;
+    try {
+        // the context's own planner, so that this is the table a context works from
+        std::vector<int64_t> heads(static_cast<size_t>(num_tensors), 0);
+        if (x0)
+            for (int32_t k = 0; k < num_tensors; ++k) heads[k] = desloc::head_elems(x0[k], numel[k]);
+        const int64_t n = desloc::count_chunks(numel, num_tensors, chunk_elems, heads.data());
+        if (cap > 0) {
+            std::vector<desloc::Chunk> chunks(static_cast<size_t>(n));
+            desloc::fill_chunks(numel, num_tensors, chunk_elems, chunks.data(), heads.data());
+            for (int64_t c = 0; c < n && c < cap; ++c) {
+                out[3 * c + 0] = chunks[c].tensor;
+                out[3 * c + 1] = chunks[c].start;
+                out[3 * c + 2] = chunks[c].count;
             }
-            ++n;
         }
+        return n;
+    } catch (const std::bad_alloc &) {
+        return DESLOC_E_NOMEM;
     }
-    return n;
+}
+
+int64_t desloc_plan_chunks(const int64_t *numel, int32_t num_tensors, int64_t chunk_elems,
+                           int64_t *out, int64_t cap) {
+    return desloc_plan_chunks_at(numel, num_tensors, chunk_elems, nullptr, out, cap);
 }
 
 int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *const *x, float *const *u,

@@ -2,7 +2,7 @@
 // worker replicas (Algorithm 1 with the Adam, ADOPT and SGDM rules of Algorithms 2-3).
 //
 // Work decomposition.  The tensor list is cut into chunks of one tensor (table built once on the
-// host); a chunk is a run of up to 8-16 tiles of tile_elems(M) elements.  A thread block takes
+// host); a chunk is a run of up to 8 tiles of tile_elems(M) elements.  A thread block takes
 // one chunk of ALL M replicas (for M = 1, and on local steps of more than eight workers, of
 // one replica) and streams its tiles through two shared-memory buffers:
 //   1. the first 4*M threads look up the chunk's pointers once; each owns one (array, worker)
@@ -29,7 +29,7 @@
 // ("copy" = the device-to-device copy bandwidth of the same GPU; these are single-tensor
 // experiments with the pointers in the kernel parameters).  In the library, with the tensor
 // list's pointer look-up on every block's path, the pipelined form is the robust one: a run
-// of 8-16 tiles per block through two buffers gives 26.1 ms (1.04) on the 218-tensor list,
+// of 8 tiles per block through two buffers gives 26.1 ms (1.04) on the 218-tensor list,
 // local and sync steps alike.
 //
 // DIAG instantiations also accumulate, from values already in registers, the squared L2 norms
@@ -55,8 +55,8 @@ constexpr int DRAIN_WAIT_LIMIT = 1 << 22;               // bound on the wait for
 // eight workers), 28-57 KB of shared memory per buffer.
 __host__ __device__ constexpr int tile_elems(int mt) { return mt <= 2 ? 1024 : 512; }
 // Tiles per chunk on large problems (one pointer look-up and one pipeline fill serve them all):
-// 8 measured best up to four workers, 16 beyond.
-__host__ __device__ constexpr int max_tiles_per_chunk(int mt) { return mt <= 4 ? 8 : 16; }
+// 8 measured best (4: sync steps 2 % slower; 16: 0.5-1 % slower; 32: 2 % slower).
+__host__ __device__ constexpr int max_tiles_per_chunk(int) { return 8; }
 
 struct __align__(16) Chunk {
     int32_t tensor;  // index into the tensor list

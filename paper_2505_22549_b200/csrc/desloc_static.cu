@@ -50,6 +50,8 @@ int32_t g_mirror_nt = 0;
 int64_t g_mirror_nptr = 0;
 int64_t g_mirror_chunk_elems = 0;
 int64_t g_mirror_numel[kMaxPointers];
+int64_t g_mirror_heads[kMaxPointers];  // short first chunk per tensor of the mirrored plan
+int64_t g_heads[kMaxPointers];         // the same for the call in progress
 
 // First call on a device: resolve the device address of the scratch array with that device
 // current.  No cudaMalloc happens here; the array is part of the module the runtime loads.
@@ -86,13 +88,15 @@ extern "C" DESLOC_API int desloc_step_static(const desloc_config *cfg, float *co
     if (cfg->M > desloc::MAX_MT) return DESLOC_E_TOO_LARGE;
     const int64_t nptr = static_cast<int64_t>(cfg->M) * cfg->num_tensors;
     if (nptr > kMaxPointers) return DESLOC_E_TOO_LARGE;
-    const int64_t chunk_elems = desloc::chunk_elems_for(cfg->M, cfg->numel, cfg->num_tensors);
-    const int64_t nchunks = desloc::count_chunks(cfg->numel, cfg->num_tensors, chunk_elems);
-    if (nchunks > kMaxChunks) return DESLOC_E_TOO_LARGE;
     for (int64_t i = 0; i < nptr; ++i) {
         if (!x[i] || !u[i] || !grads[i]) return DESLOC_E_NULL;
         if (cfg->opt != DESLOC_SGDM && !v[i]) return DESLOC_E_NULL;
     }
+    std::lock_guard<std::mutex> lock(g_mutex);
+    const int64_t chunk_elems = desloc::chunk_elems_for(cfg->M, cfg->numel, cfg->num_tensors);
+    for (int32_t k = 0; k < cfg->num_tensors; ++k) g_heads[k] = desloc::head_elems(x[k], cfg->numel[k]);
+    const int64_t nchunks = desloc::count_chunks(cfg->numel, cfg->num_tensors, chunk_elems, g_heads);
+    if (nchunks > kMaxChunks) return DESLOC_E_TOO_LARGE;
     const uint32_t mask = desloc::mask_at(cfg, t);
     const desloc::LaunchPlan plan = desloc::plan_launch(*cfg, mask, nchunks, false);
     if (!plan.fn) return DESLOC_E_INVALID;
@@ -113,7 +117,6 @@ extern "C" DESLOC_API int desloc_step_static(const desloc_config *cfg, float *co
         if (e != cudaSuccess) { rc = DESLOC_E_CUDA; break; }
         if (cap != cudaStreamCaptureStatusNone) { rc = DESLOC_E_INVALID; break; }
 
-        std::lock_guard<std::mutex> lock(g_mutex);
         void *scratch = nullptr;
         e = scratch_address(cuda_device, &scratch);
         if (e != cudaSuccess) { rc = DESLOC_E_CUDA; break; }
@@ -124,6 +127,8 @@ extern "C" DESLOC_API int desloc_step_static(const desloc_config *cfg, float *co
         const bool same_plan = same_device && g_mirror_nt == cfg->num_tensors &&
                                g_mirror_chunk_elems == chunk_elems &&
                                std::memcmp(g_mirror_numel, cfg->numel,
+                                           static_cast<size_t>(cfg->num_tensors) * sizeof(int64_t)) == 0 &&
+                               std::memcmp(g_mirror_heads, g_heads,
                                            static_cast<size_t>(cfg->num_tensors) * sizeof(int64_t)) == 0;
         const bool same_count = same_device && g_mirror_nptr == nptr;
         if (!same_device) g_mirror_device = -1;  // until the uploads below have been enqueued
@@ -132,8 +137,9 @@ extern "C" DESLOC_API int desloc_step_static(const desloc_config *cfg, float *co
         // to start at zero.  The copies are ordered before the kernel on `st`; the source is
         // pageable host memory, so each copy returns once the driver has taken the data.
         if (!same_plan) {
-            desloc::fill_chunks(cfg->numel, cfg->num_tensors, chunk_elems, g_mirror.chunks);
+            desloc::fill_chunks(cfg->numel, cfg->num_tensors, chunk_elems, g_mirror.chunks, g_heads);
             std::memcpy(g_mirror_numel, cfg->numel, static_cast<size_t>(cfg->num_tensors) * sizeof(int64_t));
+            std::memcpy(g_mirror_heads, g_heads, static_cast<size_t>(cfg->num_tensors) * sizeof(int64_t));
             g_mirror_nt = cfg->num_tensors;
             g_mirror_chunk_elems = chunk_elems;
             e = cudaMemcpyAsync(base + offsetof(ScratchImage, chunks), g_mirror.chunks,

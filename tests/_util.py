@@ -42,12 +42,19 @@ class State:
         self.u = [mk(torch.float32) for _ in range(w.M)]
         self.v = [mk(torch.float32) for _ in range(w.M)] if w.opt != "sgdm" else None
         self.g = [mk(gdt) for _ in range(w.M)]
-        for m in range(w.M):
-            self.x[m].copy_(x0)
-            if self.v is not None and v_init:
-                self.v[m].fill_(v_init)
-        del x0
+        self.v_init = v_init
         self.valid = None
+        self.reset(x0)
+
+    def reset(self, x0=None):
+        """Back to the initial state, in the same buffers."""
+        if x0 is None:
+            x0 = di.init_params(self.w, device=self.device, align=self.align)
+        for m in range(self.w.M):
+            self.x[m].copy_(x0)
+            self.u[m].zero_()
+            if self.v is not None:
+                self.v[m].fill_(self.v_init)
 
     def views(self, bufs):
         return [[b[o:o + n] for o, n in zip(self.offs, self.w.numel)] for b in bufs]

@@ -63,7 +63,7 @@ def test_sync_mask_matches_oracle_schedule(d):
 
 def test_chunk_plan_covers_every_element_once(d):
     big = [1 << 24] * 4                       # plenty of tiles: the full run per chunk
-    want = {1: 8192, 2: 8192, 3: 4096, 4: 4096, 5: 8192, 8: 8192, 9: 8192, 256: 8192}
+    want = {1: 8192, 2: 8192, 3: 4096, 4: 4096, 5: 4096, 8: 4096, 9: 8192, 256: 8192}
     for M, ce_want in want.items():
         assert d.desloc_chunk_elems(d.make_config(M, big, "adam", "bf16")) == ce_want
     # a small problem gets single-tile chunks so that it still spreads over many blocks
@@ -92,6 +92,39 @@ def test_chunk_plan_covers_every_element_once(d):
     with pytest.raises(d.DeslocError) as e:
         d.desloc_plan_chunks([5, 0], ce)
     assert e.value.status == d.DESLOC_E_RANGE
+
+
+def test_chunk_plan_cuts_first_chunks_at_2kb_boundaries(d):
+    """With the addresses of worker 0's x tensors the plan shortens a tensor's first chunk so
+    that all later ones start on a 2 KB boundary -- where the address allows it (a multiple of
+    32 bytes) and the tensor reaches the boundary."""
+    ce = 4096
+    base = 0x7f0000000000                     # 2 KB aligned
+    numel = [10_000, 10_000, 10_000, 10_000, 300, 10_000, 3 * ce + 512 - 64]
+    addr = [base, base + 4 * 64, base + 4 * 504, base + 4 * 4, base + 4 * 448, base + 2048,
+            base + 4 * 64]
+    total, chunks = d.desloc_plan_chunks(numel, ce, x0=addr)
+    per = {k: [(s, c) for kk, s, c in chunks if kk == k] for k in range(len(numel))}
+    assert per[0][0] == (0, ce)                            # on the boundary: nothing cut
+    assert per[1][0] == (0, 448) and per[1][1] == (448, ce)
+    assert per[2][0] == (0, 8) and per[2][1] == (8, ce)
+    assert per[3][0] == (0, ce)                            # 16 bytes off: not a multiple of 32
+    assert per[4] == [(0, 64), (64, 236)]                  # short tensor that crosses the boundary
+    assert per[5][0] == (0, ce)
+    assert per[6] == [(0, 448), (448, ce), (448 + ce, ce), (448 + 2 * ce, ce)]
+    for k, lst in per.items():
+        pos = 0
+        for s, c in lst:
+            assert s == pos and c >= 1
+            pos += c
+            if s > 0 and addr[k] % 32 == 0:
+                assert (addr[k] + 4 * s) % 2048 == 0
+        assert pos == numel[k]
+    assert total == len(chunks)
+    # a tensor that ends in front of the boundary stays whole
+    assert d.desloc_plan_chunks([60], ce, x0=[base + 4 * 448])[1] == [(0, 0, 60)]
+    # no addresses: the plain plan
+    assert d.desloc_plan_chunks(numel, ce)[1] == d.desloc_plan_chunks(numel, ce, x0=[base] * len(numel))[1]
 
 
 def test_workload_sizes_match_the_stated_totals():
