@@ -322,9 +322,9 @@ DESLOC_API int64_t desloc_chunk_elems(const desloc_config *cfg);
  * not survive a cudaDeviceReset().
  *
  * Uploads.  The library keeps a host copy of what it last wrote into the array.  A call
- * uploads only the tables that differ from it (the chunk table depends on the tensor list
- * alone, the four pointer tables on x, u, v, grads), from ordinary pageable host memory,
- * ahead of the kernel on `stream`; such a copy may wait for work already enqueued on `stream`
+ * uploads only the tables that differ from it (the chunk table depends on the tensor list and
+ * the alignment of worker 0's x, the four pointer tables on x, u, v, grads), from ordinary
+ * pageable host memory, ahead of the kernel on `stream`; such a copy may wait for work already enqueued on `stream`
  * before it returns.  A loop that steps the same buffers every time uploads nothing after its
  * first call and only enqueues the kernel.  Because those copies read host memory the library
  * reuses, the call returns DESLOC_E_INVALID, enqueueing nothing, while `stream` is being

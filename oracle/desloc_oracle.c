@@ -227,9 +227,9 @@ uint32_t desloc_oracle_step(const desloc_oracle_cfg *c, int64_t t, double lr, do
 }
 
 /*
- * Norm-based gradient clipping, the form the paper's language-model runs used (model table:
- * "norm-based gradient clipping with clip-bound rho"): worker m's whole gradient (all tensors,
- * here one [M][stride] array) is scaled by min(1, max_norm / ||g^m||_2).  Writes the norms and
+ * Clipping by the gradient's norm, the form the paper's language-model runs used (the model
+ * table of the experimental-details appendix lists it with the bound rho): worker m's whole
+ * gradient (all tensors, here one [M][stride] array) is scaled by min(1, max_norm / ||g^m||_2).  Writes the norms and
  * the factors; a zero gradient keeps factor 1.
  */
 void desloc_oracle_norm_scales(int32_t M, int64_t n, int64_t stride, const float *g, double max_norm,
