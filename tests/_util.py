@@ -29,19 +29,22 @@ class State:
     """Per-worker flat fp32 buffers x, u, v and gradient buffer g on `device`, plus per-tensor views."""
 
     def __init__(self, w: di.Workload, device, align: int = 4, byte_shift: int = 0,
-                 v_init: float = 0.0):
+                 v_init: float = 0.0, g_shift: int | None = None):
         self.w, self.device, self.align = w, device, align
         self.offs = di.offsets_of(w.numel, align)
         self.nflat = di.flat_size(w.numel, align)
         gdt = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
         x0 = di.init_params(w, device=device, align=align)
-        # byte_shift (in elements) moves every buffer off its natural 16-byte alignment
+        # byte_shift (in elements) moves every buffer off its natural alignment (g_shift: the
+        # gradient buffers by another amount than the state)
         sh = byte_shift
         mk = lambda dt: torch.zeros(self.nflat + sh, dtype=dt, device=device)[sh:]
+        gsh = byte_shift if g_shift is None else g_shift
+        mkg = lambda dt: torch.zeros(self.nflat + gsh, dtype=dt, device=device)[gsh:]
         self.x = [mk(torch.float32) for _ in range(w.M)]
         self.u = [mk(torch.float32) for _ in range(w.M)]
         self.v = [mk(torch.float32) for _ in range(w.M)] if w.opt != "sgdm" else None
-        self.g = [mk(gdt) for _ in range(w.M)]
+        self.g = [mkg(gdt) for _ in range(w.M)]
         self.v_init = v_init
         self.valid = None
         self.reset(x0)

@@ -34,11 +34,11 @@ def make_engine(d, w, st, post=False):
 
 
 def run_both(w, T, align=4, byte_shift=0, post=False, v_init=0.0, identical=False,
-             forced_masks=None, lr_of_t=None, max_blocks=0):
+             forced_masks=None, lr_of_t=None, max_blocks=0, g_shift=None):
     """Runs T steps on the GPU and in the oracle on identical inputs; returns both end states."""
     d = _lib()
     dev = torch.device("cuda:0")
-    st = State(w, dev, align=align, byte_shift=byte_shift, v_init=v_init)
+    st = State(w, dev, align=align, byte_shift=byte_shift, v_init=v_init, g_shift=g_shift)
     eng = make_engine(d, w, st, post)
     if max_blocks:
         d.desloc_testing_set_max_blocks(eng.ctx, max_blocks)   # blocks stride over the chunks
@@ -166,6 +166,21 @@ def test_misaligned_buffers_take_the_scalar_path():
     for shift in (1, 2, 3):
         res = run_both(w, 6, align=1, byte_shift=shift)
         check(res)
+
+
+@pytest.mark.parametrize("M,opt", [(2, "adam"), (4, "adopt"), (8, "sgdm"), (12, "adam")])
+@pytest.mark.parametrize("shift,g_shift", [(8, None), (24, None), (504, None), (8, 0), (8, 4), (40, 16)])
+def test_first_chunks_cut_at_2kb_boundaries(M, opt, shift, g_shift):
+    """State buffers that start 32 B ... 2016 B past a 2 KB boundary: the chunk plan cuts every
+    tensor's first chunk at the next boundary (504, 488, 8 elements here, and others for the
+    later tensors).  Gradients that share the state's offsets are then aligned as well; gradients
+    laid out differently (g_shift) stay 16-byte aligned where they were (shift 0, 16 elements)
+    or take the scalar path (bf16 shifted by 4 elements = 8 bytes)."""
+    gd = "bf16" if opt != "sgdm" else "f32"
+    w = di.Workload("heads", opt, M, (512 * 9 + 64, 40, 1024, 512 * 3 - 8, 7), gd, "normal1", lr=1e-2,
+                    K=(2, 3, 4), seed=11, adopt_norm_clip=(opt == "adopt"))
+    res = run_both(w, 7, align=8, byte_shift=shift, g_shift=g_shift)
+    check(res)
 
 
 # ------------------------------------------------------------------ scaled-down paper workloads
