@@ -4,6 +4,7 @@ before any CUDA call."""
 import os
 import re
 
+import numpy as np
 import pytest
 
 import desloc_inputs as di
@@ -127,6 +128,41 @@ def test_chunk_plan_cuts_first_chunks_at_2kb_boundaries(d):
     assert d.desloc_plan_chunks([60], ce, x0=[base + 4 * 448])[1] == [(0, 0, 60)]
     # no addresses: the plain plan
     assert d.desloc_plan_chunks(numel, ce)[1] == d.desloc_plan_chunks(numel, ce, x0=[base] * len(numel))[1]
+
+
+def test_chunk_plan_at_random_addresses_covers_every_element_once(d):
+    """Seeded sweep over tensor lists and addresses (any 4-byte alignment): every element of
+    every tensor lies in exactly one chunk, chunks of a tensor are contiguous and in order, only
+    the first and the last are short, and the later ones start on 2 KB boundaries unless the
+    address is of the one kind the plan leaves alone."""
+    rng = np.random.default_rng(2505)
+    for trial in range(200):
+        nt = int(rng.integers(1, 12))
+        ce = int(rng.choice([512, 1024, 4096, 8192]))
+        numel = [int(rng.choice([1, 7, 500, 511, 512, 513, 4096, 9000, 40_000])) + int(rng.integers(0, 3))
+                 for _ in range(nt)]
+        addr = [0x7f0000000000 + 4 * int(rng.integers(0, 4096)) for _ in range(nt)]
+        total, chunks = d.desloc_plan_chunks(numel, ce, x0=addr)
+        assert total == len(chunks)
+        pos = [0] * nt
+        first = [True] * nt
+        last_k = -1
+        for k, s0, c in chunks:
+            assert k >= last_k                   # tensors in order
+            last_k = k
+            assert s0 == pos[k] and 1 <= c <= ce
+            left = numel[k] - s0
+            if first[k]:
+                cut = (512 - (addr[k] // 4) % 512) % 512
+                leaves_alone = addr[k] % 32 == 16 or cut == 0 or cut >= numel[k]
+                assert c == (min(ce, left) if leaves_alone else cut)
+            else:
+                assert c == min(ce, left)
+                if addr[k] % 32 != 16:
+                    assert (addr[k] + 4 * s0) % 2048 == 0
+            first[k] = False
+            pos[k] += c
+        assert pos == numel
 
 
 def test_workload_sizes_match_the_stated_totals():
