@@ -275,9 +275,9 @@ DESLOC_API int64_t desloc_get_launch_count(const desloc_ctx *ctx);
  *        alignment at all.  So a tensor that does not start on a 2 KB boundary has its first
  *        chunk cut to the elements in front of the next one, and every later chunk starts on
  *        it -- for x and for every array laid out like x (the same element offsets in a
- *        buffer of its own).  The one exception is an address that is a multiple of 16 but not
- *        of 32 bytes, which is left alone (the cut would be an odd multiple of 4 elements and
- *        could move an independently laid out bf16 gradient off its 16-byte alignment).
+ *        buffer of its own).  A gradient laid out differently may end up 8 or 2 bytes off a
+ *        16-byte boundary after the cut; such chunks are updated straight from global memory
+ *        (128-bit accesses, or coordinate by coordinate), correctly but more slowly.
  * desloc_plan_chunks_at() with the x pointers given to desloc_create() is the table that context
  * works from; desloc_plan_chunks() is the same with x0 = NULL.
  */

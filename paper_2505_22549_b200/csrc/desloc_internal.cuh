@@ -99,14 +99,16 @@ inline int64_t chunk_elems_for(int32_t M, const int64_t *numel, int32_t num_tens
 // every later chunk of it starts on a 2 KB boundary of worker 0's x -- and with it of every
 // array that shares x's element offsets, the usual layout (one flat buffer per worker and array).
 // The same cut turns a tensor that starts at an odd offset of a tightly packed buffer (x not
-// even 16-byte aligned: every chunk of it would take the scalar path) into a short scalar head
-// and an aligned rest.  One case is left alone: x 16-byte but not 32-byte aligned.  There the
-// cut is an odd multiple of 4 elements, which would move a bf16 gradient that does NOT share
-// x's offsets off the 16-byte alignment it has now.
+// 16-byte aligned: every chunk of it would take the scalar path), or at an odd multiple of four
+// elements of a buffer padded to 16 bytes (x aligned, a bf16 gradient with the same offsets
+// 8 bytes off), into a short head and an aligned rest.  A gradient that does NOT share x's
+// offsets can lose its 16-byte alignment by the cut; where it keeps 8 bytes, the chunk is
+// updated with 128-bit accesses from global memory (0.66-0.86 of the copy bandwidth), else
+// coordinate by coordinate.
 constexpr int64_t ALIGN_PHASE_ELEMS = 512;
 inline int64_t head_elems(const void *x0, int64_t numel) {
     const uintptr_t a = reinterpret_cast<uintptr_t>(x0);
-    if ((a & 3u) != 0 || (a & 31u) == 16u) return 0;
+    if ((a & 3u) != 0) return 0;
     const int64_t phase = static_cast<int64_t>(a >> 2) & (ALIGN_PHASE_ELEMS - 1);
     const int64_t head = (ALIGN_PHASE_ELEMS - phase) & (ALIGN_PHASE_ELEMS - 1);
     return head < numel ? head : 0;

@@ -320,6 +320,19 @@ struct GlobalAcc {
     __device__ __forceinline__ FV<1> ldg(int m, int q) const { return ld_grad<1, GT>(sp[3][m], q); }
 };
 
+// The same with four coordinates per position and 128-bit accesses (64-bit for bf16 gradients):
+// chunks whose fp32 arrays are 16-byte aligned while the bf16 gradients are only 8-byte aligned
+// -- a flat layout padded to 16 bytes, where the gradient of a tensor at an odd multiple of
+// four elements sits 8 bytes off -- and the aligned part of a ragged last tile.
+template <int MT, typename GT>
+struct GlobalAcc4 {
+    static constexpr int VEC = 4;
+    char *const (*sp)[MT];
+    __device__ __forceinline__ FV<4> ld(int arr, int m, int q) const { return ld_f32<4>(sp[arr][m], 4LL * q); }
+    __device__ __forceinline__ void st(int arr, int m, int q, const FV<4> &r) const { st_f32<4>(sp[arr][m], 4LL * q, r); }
+    __device__ __forceinline__ FV<4> ldg(int m, int q) const { return ld_grad<4, GT>(sp[3][m], 4LL * q); }
+};
+
 // ---- diagnostics ------------------------------------------------------------------------------
 // Each thread keeps its own running sums of squares, one per (kind, worker), in registers over
 // all tiles of a chunk.  At the end of the chunk a warp reduces each of them (shuffle tree) into
@@ -576,6 +589,9 @@ desloc_step_kernel(const __grid_constant__ StepArgs a) {
         // is a multiple of 16 (only the chunk's last tile can miss that: it is then updated
         // straight from global memory, like every tile of a chunk whose pointers are unaligned)
         const bool unaligned = __syncthreads_or((reinterpret_cast<uintptr_t>(p) & 15u) != 0) != 0;
+        // 128-bit accesses from global memory need less: 8 bytes for bf16 gradients
+        const uintptr_t need = (arr == 3 && sizeof(GT) == 2) ? 7u : 15u;
+        const bool wide_ok = __syncthreads_or((reinterpret_cast<uintptr_t>(p) & need) != 0) == 0;
         const int ntiles = (count + T - 1) / T;
         const int staged = unaligned ? 0 : ((count % T) % ALIGN_ELEMS == 0 ? ntiles : ntiles - 1);   // tiles 0 .. staged-1
         // request tile k (< staged) into its buffer: every owner its own slice, one arrival
@@ -626,7 +642,14 @@ desloc_step_kernel(const __grid_constant__ StepArgs a) {
         }
         if (staged * T < count) {
             // what could not be staged: the whole chunk, or its ragged last tile
-            const int e0 = staged * T;
+            int e0 = staged * T;
+            if (wide_ok) {
+                const GlobalAcc4<MT, GT> acc4{sp};
+                const int p1 = count >> 2;
+                for (int q = (e0 >> 2) + tid; q < p1; q += BLOCK_THREADS)
+                    update_position<OPT, MASK, MT, POST, DIAG>(a, acc4, sscale, q, wn);
+                e0 = p1 << 2;
+            }
             const GlobalAcc<MT, GT> acc{sp};
             for (int e = e0 + tid; e < count; e += BLOCK_THREADS)
                 update_position<OPT, MASK, MT, POST, DIAG>(a, acc, sscale, e, wn);

@@ -97,8 +97,7 @@ def test_chunk_plan_covers_every_element_once(d):
 
 def test_chunk_plan_cuts_first_chunks_at_2kb_boundaries(d):
     """With the addresses of worker 0's x tensors the plan shortens a tensor's first chunk so
-    that all later ones start on a 2 KB boundary -- unless the address is a multiple of 16 but
-    not of 32 bytes, or the tensor ends in front of the boundary."""
+    that all later ones start on a 2 KB boundary -- unless the tensor ends in front of it."""
     ce = 4096
     base = 0x7f0000000000                     # 2 KB aligned
     numel = [10_000, 10_000, 10_000, 10_000, 300, 10_000, 3 * ce + 512 - 64, 10_000, 10_000]
@@ -109,7 +108,7 @@ def test_chunk_plan_cuts_first_chunks_at_2kb_boundaries(d):
     assert per[0][0] == (0, ce)                            # on the boundary: nothing cut
     assert per[1][0] == (0, 448) and per[1][1] == (448, ce)
     assert per[2][0] == (0, 8) and per[2][1] == (8, ce)
-    assert per[3][0] == (0, ce)                            # 16 bytes off a multiple of 32: left alone
+    assert per[3][0] == (0, 508) and per[3][1] == (508, ce)   # an odd multiple of four elements
     assert per[7][0] == (0, 507) and per[7][1] == (507, ce)   # an odd offset of a packed buffer
     assert per[8][0] == (0, 2) and per[8][1] == (2, ce)
     assert per[4] == [(0, 64), (64, 236)]                  # short tensor that crosses the boundary
@@ -120,7 +119,7 @@ def test_chunk_plan_cuts_first_chunks_at_2kb_boundaries(d):
         for s, c in lst:
             assert s == pos and c >= 1
             pos += c
-            if s > 0 and addr[k] % 32 != 16:
+            if s > 0:
                 assert (addr[k] + 4 * s) % 2048 == 0
         assert pos == numel[k]
     assert total == len(chunks)
@@ -133,8 +132,7 @@ def test_chunk_plan_cuts_first_chunks_at_2kb_boundaries(d):
 def test_chunk_plan_at_random_addresses_covers_every_element_once(d):
     """Seeded sweep over tensor lists and addresses (any 4-byte alignment): every element of
     every tensor lies in exactly one chunk, chunks of a tensor are contiguous and in order, only
-    the first and the last are short, and the later ones start on 2 KB boundaries unless the
-    address is of the one kind the plan leaves alone."""
+    the first and the last are short, and the later ones start on 2 KB boundaries."""
     rng = np.random.default_rng(2505)
     for trial in range(200):
         nt = int(rng.integers(1, 12))
@@ -154,12 +152,11 @@ def test_chunk_plan_at_random_addresses_covers_every_element_once(d):
             left = numel[k] - s0
             if first[k]:
                 cut = (512 - (addr[k] // 4) % 512) % 512
-                leaves_alone = addr[k] % 32 == 16 or cut == 0 or cut >= numel[k]
+                leaves_alone = cut == 0 or cut >= numel[k]
                 assert c == (min(ce, left) if leaves_alone else cut)
             else:
                 assert c == min(ce, left)
-                if addr[k] % 32 != 16:
-                    assert (addr[k] + 4 * s0) % 2048 == 0
+                assert (addr[k] + 4 * s0) % 2048 == 0
             first[k] = False
             pos[k] += c
         assert pos == numel

@@ -169,13 +169,14 @@ def test_misaligned_buffers_take_the_scalar_path():
 
 
 @pytest.mark.parametrize("M,opt", [(2, "adam"), (4, "adopt"), (8, "sgdm"), (12, "adam")])
-@pytest.mark.parametrize("shift,g_shift", [(8, None), (24, None), (504, None), (8, 0), (8, 4), (40, 16)])
+@pytest.mark.parametrize("shift,g_shift", [(8, None), (24, None), (504, None), (8, 0), (8, 4), (40, 16),
+                                           (4, None), (4, 0), (12, 2), (1, None), (3, 0)])
 def test_first_chunks_cut_at_2kb_boundaries(M, opt, shift, g_shift):
     """State buffers that start 32 B ... 2016 B past a 2 KB boundary: the chunk plan cuts every
     tensor's first chunk at the next boundary (504, 488, 8 elements here, and others for the
     later tensors).  Gradients that share the state's offsets are then aligned as well; gradients
     laid out differently (g_shift) stay 16-byte aligned where they were (shift 0, 16 elements)
-    or take the scalar path (bf16 shifted by 4 elements = 8 bytes)."""
+    or take the 128-bit path from global memory (bf16 shifted by 4 elements = 8 bytes)."""
     gd = "bf16" if opt != "sgdm" else "f32"
     w = di.Workload("heads", opt, M, (512 * 9 + 64, 40, 1024, 512 * 3 - 8, 7), gd, "normal1", lr=1e-2,
                     K=(2, 3, 4), seed=11, adopt_norm_clip=(opt == "adopt"))
