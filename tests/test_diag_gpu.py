@@ -38,12 +38,13 @@ def _check_norms(st, got_per, got_tot, arrays, what):
                                     ("cfg5_adam_desloc", 5), ("cfg2_adam_135m", 12),
                                     ("cfg3_adopt_360m", 11), ("cfg5_sgdm_desloc", 2)])
 @pytest.mark.parametrize("post", [False, True])
-@pytest.mark.parametrize("align", [4, 1])
-def test_diag_step_norms_match_oracle_and_state_matches_plain_step(name, M, post, align):
+@pytest.mark.parametrize("align,g_shift", [(4, None), (1, None), (8, 4)])
+def test_diag_step_norms_match_oracle_and_state_matches_plain_step(name, M, post, align, g_shift):
     import paper_2505_22549_b200 as d
     w = di.mini(di.WORKLOADS[name], T=9).replace(M=M, K=(2, 3, 4))
     dev = torch.device("cuda:0")
-    a, b = State(w, dev, align=align), State(w, dev, align=align)    # diag / plain
+    # (g_shift: gradients 8 bytes off the state's layout -- the 128-bit path from global memory)
+    a, b = State(w, dev, align=align, g_shift=g_shift), State(w, dev, align=align, g_shift=g_shift)    # diag / plain
     ea, eb = make_engine(d, w, a, post), make_engine(d, w, b, post)
     ox, ou = a.to_numpy(a.x), a.to_numpy(a.u)
     ov = a.to_numpy(a.v) if a.v is not None else None
