@@ -253,6 +253,12 @@ def timed_loop(stream, fn, reps):
     return e0.elapsed_time(e1) / reps
 
 
+def timed_median(stream, fn, steps=20, repeats=5):
+    """Median (and spread) over `repeats` CUDA-event timings of `steps` back-to-back calls."""
+    ms = sorted(timed_loop(stream, fn, steps) for _ in range(repeats))
+    return ms[len(ms) // 2], {"ms_min": ms[0], "ms_max": ms[-1], "steps_per_repeat": steps, "repeats": repeats}
+
+
 def rates(w, ms, peak, nbytes=None):
     nbytes = nbytes if nbytes is not None else w.M * w.N * bytes_per_param(w)
     gbs = nbytes / (ms * 1e-3) / 1e9
@@ -261,24 +267,28 @@ def rates(w, ms, peak, nbytes=None):
 
 
 def per_mask_and_variants(w, eng, g, stream, peak, reps):
-    """Local, x-only and all-sync steps timed in isolation, then the norm-clipped step (one more
-    read of the gradients) and the diagnostics step (same bytes as the plain step)."""
+    """Local, x-only and all-sync steps timed in isolation (median of five timings of at least
+    twenty back-to-back steps of the same mask), then the norm-clipped step (one more read of the
+    gradients) and the diagnostics step (same bytes as the plain step)."""
     out = {"by_mask": {}}
     for mk in [0, 1, 3 if w.opt == "sgdm" else 7]:
         if w.M == 1 and mk:
             continue
         fn = lambda: eng.step_masked(mk, w.lr, g, clip_bound=1.0)
         fn(); fn()
-        out["by_mask"][str(mk)] = rates(w, timed_loop(stream, fn, reps), peak)
+        ms, spread = timed_median(stream, fn, steps=max(reps, 20), repeats=5)
+        out["by_mask"][str(mk)] = dict(rates(w, ms, peak), **spread)
     gbytes = 2 if w.grad_dtype == "bf16" else 4
     fn = lambda: eng.step_normclip(1, w.lr, g, 1.0, clip_bound=1.0)
     fn(); fn()
     nc_bytes = w.M * w.N * (bytes_per_param(w) + gbytes)
-    out["normclip_step"] = dict(rates(w, timed_loop(stream, fn, reps), peak, nc_bytes),
-                                launches_per_step=3, algorithmic_bytes=nc_bytes)
+    ms, spread = timed_median(stream, fn, steps=max(reps, 20), repeats=3)
+    out["normclip_step"] = dict(rates(w, ms, peak, nc_bytes), launches_per_step=3,
+                                algorithmic_bytes=nc_bytes, **spread)
     fn = lambda: eng.step_diag(1, w.lr, g, clip_bound=1.0)
     fn(); fn()
-    out["diag_step"] = dict(rates(w, timed_loop(stream, fn, reps), peak),
+    ms, spread = timed_median(stream, fn, steps=max(reps, 20), repeats=3)
+    out["diag_step"] = dict(rates(w, ms, peak), **spread,
                             note="same step, plus per-(worker, tensor) norms of g, x, d fused in")
     return out
 
