@@ -21,6 +21,15 @@ extern "C" {
 DESLOC_API int desloc_testing_set_max_blocks(desloc_ctx *ctx, int64_t max_blocks);
 
 /*
+ * Whether the step kernels stage their tiles through shared memory: -1 = the library decides (the
+ * default: a launch of at most two blocks per SM of single-tile chunks skips the staging, since
+ * it has nothing to overlap), 0 = stage whenever alignment allows, 1 = never (every chunk is
+ * updated straight from global memory).  Results do not depend on it.  DESLOC_E_RANGE for other
+ * values.
+ */
+DESLOC_API int desloc_testing_set_staging(desloc_ctx *ctx, int32_t mode);
+
+/*
  * How often a thread block polls for its tile's copies before it gives up (default: about four
  * million polls).  polls = 0 makes every block give up at once: the step then stores nothing,
  * the blocks still let their copies land before they leave, and every later step call returns

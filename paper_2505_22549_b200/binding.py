@@ -107,6 +107,8 @@ _lib.desloc_get_diag_norms.argtypes = [_P, ctypes.POINTER(ctypes.c_float),
                                        ctypes.POINTER(ctypes.c_float), _P]
 _lib.desloc_testing_set_max_blocks.restype = ctypes.c_int
 _lib.desloc_testing_set_max_blocks.argtypes = [_P, ctypes.c_int64]
+_lib.desloc_testing_set_staging.restype = ctypes.c_int
+_lib.desloc_testing_set_staging.argtypes = [_P, ctypes.c_int32]
 _lib.desloc_testing_set_wait_limit.restype = ctypes.c_int
 _lib.desloc_testing_set_wait_limit.argtypes = [_P, ctypes.c_int32]
 _lib.desloc_plan_chunks.restype = ctypes.c_int64
@@ -316,6 +318,13 @@ def desloc_chunk_elems(cfg: DeslocConfig) -> int:
     if n < 0:
         raise DeslocError(n, "desloc_chunk_elems")
     return n
+
+
+def desloc_testing_set_staging(ctx: int, mode: int) -> None:
+    """Test hook (include/desloc_testing.h): -1 the library decides, 0 always stage, 1 never."""
+    rc = _lib.desloc_testing_set_staging(ctx, int(mode))
+    if rc != DESLOC_OK:
+        raise DeslocError(rc, "desloc_testing_set_staging")
 
 
 def desloc_testing_set_wait_limit(ctx: int, polls: int) -> None:

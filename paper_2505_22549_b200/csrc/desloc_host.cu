@@ -192,6 +192,7 @@ struct desloc_ctx {
     int last_cuda_error = 0;
     bool diag_valid = false;        // a diagnostics step has run since the workers last changed
     int64_t max_blocks = 0;         // test hook: cap on the grid (0 = one block per work item)
+    int staging_mode = -1;          // test hook: -1 the library decides, 0 always stage, 1 never
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t ev_entry = nullptr;
     cudaEvent_t ev_group[kHostGroups] = {};
@@ -332,6 +333,7 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
         desloc::fill_hyper(a, c, lr_t, clip_bound_t);
         a.err = ctx->d_err;
         a.wait_limit = ctx->wait_limit;
+        a.direct = ctx->staging_mode < 0 ? (plan.direct ? 1 : 0) : ctx->staging_mode;
 
         void *params[] = {&a};
         const auto capped = [ctx](const desloc::LaunchPlan &lp) {
@@ -757,6 +759,13 @@ int desloc_testing_set_max_blocks(desloc_ctx *ctx, int64_t max_blocks) {
     if (!ctx) return DESLOC_E_NULL;
     if (max_blocks < 0) return DESLOC_E_RANGE;
     ctx->max_blocks = max_blocks;
+    return DESLOC_OK;
+}
+
+int desloc_testing_set_staging(desloc_ctx *ctx, int32_t mode) {
+    if (!ctx) return DESLOC_E_NULL;
+    if (mode < -1 || mode > 1) return DESLOC_E_RANGE;
+    ctx->staging_mode = mode;
     return DESLOC_OK;
 }
 

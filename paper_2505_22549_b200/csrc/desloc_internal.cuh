@@ -175,6 +175,7 @@ inline void fill_hyper(StepArgs &a, const desloc_config &c, float lr_t, float cl
                                                        : std::numeric_limits<float>::infinity();
     a.wait_limit = DEFAULT_WAIT_LIMIT;
     a.err = nullptr;
+    a.direct = 0;
 }
 
 // Which kernel a step of this configuration runs, and over how many blocks.
@@ -183,7 +184,13 @@ struct LaunchPlan {
     long long grid = 0;
     bool strides = true;  // a smaller grid may stride over the work items (not the runtime-M kernel)
     int smem = 0;         // dynamic shared memory of the launch
+    bool direct = false;  // too small to gain from staging: update straight from global memory
 };
+
+// Launches of at most this many blocks of single-tile chunks (two per SM of a B200: one wave)
+// skip the staging.  Measured on the 4096-parameter, two-worker workload: 3.08 us per step in a
+// CUDA graph of 16 steps against 3.34 us staged.
+constexpr long long DIRECT_GRID = 2 * 148;
 
 // The tile kernels use more than the 48 KB of shared memory a kernel gets by default: raise the
 // function's limit to what the launch asks for.  Not an allocation.
@@ -205,6 +212,9 @@ inline LaunchPlan plan_launch(const desloc_config &c, uint32_t mask, long long n
     p.strides = !generic;
     p.smem = generic ? 0 : step_smem_bytes(c.opt, per_worker_items ? 1 : c.M, bf16);
     p.grid = per_worker_items ? nchunks * c.M : nchunks;
+    const int mt = per_worker_items ? 1 : c.M;
+    p.direct = p.grid <= DIRECT_GRID && mt <= MAX_MT &&
+               chunk_elems_for(c.M, c.numel, c.num_tensors) == tile_elems(mt);
     return p;
 }
 

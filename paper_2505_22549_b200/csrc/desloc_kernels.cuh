@@ -81,6 +81,7 @@ struct StepArgs {
     long long diag_chunk0;  // index of chunks[0] within the context's chunk table
     int *err;             // set to 1 when a bounded wait ran out (may be nullptr)
     int wait_limit;       // iterations a block polls for its tile before it gives up
+    int direct;           // non-zero: no staging, every chunk straight from global memory (tiny launches)
     int nt;
     int M;
     float b1, omb1;   // beta1, 1 - beta1
@@ -594,7 +595,9 @@ desloc_step_kernel(const __grid_constant__ StepArgs a) {
         const uintptr_t need = (arr == 3 && sizeof(GT) == 2) ? 7u : 15u;
         const bool wide_ok = __syncthreads_or((reinterpret_cast<uintptr_t>(p) & need) != 0) == 0;
         const int ntiles = (count + T - 1) / T;
-        const int staged = unaligned ? 0 : ((count % T) % ALIGN_ELEMS == 0 ? ntiles : ntiles - 1);   // tiles 0 .. staged-1
+        // (a launch of a single wave of single-tile chunks has nothing to overlap: staging would
+        // only add the copy engine's round trip to every step of a latency-bound problem)
+        const int staged = (unaligned || a.direct) ? 0 : ((count % T) % ALIGN_ELEMS == 0 ? ntiles : ntiles - 1);   // tiles 0 .. staged-1
         // request tile k (< staged) into its buffer: every owner its own slice, one arrival
         auto request = [&](int k) {
             const int cnt = min(T, count - k * T);

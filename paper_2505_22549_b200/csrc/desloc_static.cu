@@ -177,6 +177,7 @@ extern "C" DESLOC_API int desloc_step_static(const desloc_config *cfg, float *co
         a.gscale = nullptr;
         a.diag = nullptr;
         desloc::fill_hyper(a, *cfg, lr_t, clip_bound_t);
+        a.direct = plan.direct ? 1 : 0;
         void *params[] = {&a};
         e = desloc::prepare_launch(plan);
         if (e == cudaSuccess)

@@ -230,6 +230,7 @@ def test_diag_entry_points_reject_bad_arguments_without_a_device(d):
     assert L.desloc_step_diag(None, 0, 0.1, 0.0, 0.0, None, None, None) == d.DESLOC_E_NULL
     assert L.desloc_get_diag_norms(None, None, None, None) == d.DESLOC_E_NULL
     assert L.desloc_testing_set_max_blocks(None, 0) == d.DESLOC_E_NULL
+    assert L.desloc_testing_set_staging(None, 0) == d.DESLOC_E_NULL
 
 
 STATIC_BAD = [

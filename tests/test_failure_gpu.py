@@ -26,6 +26,7 @@ def test_a_wait_that_runs_out_is_reported_and_nothing_is_stored(name):
     torch.cuda.synchronize()
     before = [st.to_numpy(b) for b in (st.x, st.u) + ((st.v,) if st.v is not None else ())]
 
+    d.desloc_testing_set_staging(eng.ctx, 0)                # stage even if the launch is small
     d.desloc_testing_set_wait_limit(eng.ctx, 0)             # every block gives up at once
     st.fill_grads(1)
     eng.step(1, f32r(w.lr), st.views(st.g), clip_bound=1.0)  # enqueues; the failure is on the device

@@ -34,7 +34,7 @@ def make_engine(d, w, st, post=False):
 
 
 def run_both(w, T, align=4, byte_shift=0, post=False, v_init=0.0, identical=False,
-             forced_masks=None, lr_of_t=None, max_blocks=0, g_shift=None):
+             forced_masks=None, lr_of_t=None, max_blocks=0, g_shift=None, staging=None):
     """Runs T steps on the GPU and in the oracle on identical inputs; returns both end states."""
     d = _lib()
     dev = torch.device("cuda:0")
@@ -42,6 +42,8 @@ def run_both(w, T, align=4, byte_shift=0, post=False, v_init=0.0, identical=Fals
     eng = make_engine(d, w, st, post)
     if max_blocks:
         d.desloc_testing_set_max_blocks(eng.ctx, max_blocks)   # blocks stride over the chunks
+    if staging is not None:
+        d.desloc_testing_set_staging(eng.ctx, staging)         # 0: always stage, 1: never
     ox, ou = st.to_numpy(st.x), st.to_numpy(st.u)
     ov = st.to_numpy(st.v) if st.v is not None else None
     ocfg = oracle_cfg(w, oracle.FLAG_POST_AVERAGE if post else 0)
@@ -99,8 +101,12 @@ def test_cfg1_adam_n4096_full_run():
 @pytest.mark.parametrize("opt", ["adam", "adopt", "sgdm"])
 @pytest.mark.parametrize("M", [1, 2, 3, 4, 5, 6, 7, 8])
 @pytest.mark.parametrize("gd", ["f32", "bf16"])
-def test_every_mask_on_ragged_tensors(opt, M, gd):
-    """Tensors of 1..9 elements, one chunk + 1, odd sizes; all 8 sync patterns in turn, twice."""
+@pytest.mark.parametrize("staging", [0, 1])
+def test_every_mask_on_ragged_tensors(opt, M, gd, staging):
+    """Tensors of 1..9 elements, one chunk + 1, odd sizes; all 8 sync patterns in turn, twice.
+    A problem this small would skip the staging by itself: it is run staged (tiles through
+    shared memory wherever alignment allows) and unstaged (everything straight from global
+    memory)."""
     numel = (1, 2, 3, 4, 5, 7, 8, 9, 4095, 4096, 4097, 8191, 12289, 31)
     nmask = 4 if opt == "sgdm" else 8
     masks = list(range(nmask)) * 2
@@ -108,8 +114,20 @@ def test_every_mask_on_ragged_tensors(opt, M, gd):
                     eps=1e-3 if opt != "adopt" else 1e-2, lr=1e-2, weight_decay=0.05,
                     clip_rho=1.5, adopt_norm_clip=(opt == "adopt"), seed=M)
     for align in (4, 1):   # 4: vector path with tails; 1: packed, odd offsets -> scalar path
-        res = run_both(w, len(masks), align=align, forced_masks=masks, v_init=0.25)
+        res = run_both(w, len(masks), align=align, forced_masks=masks, v_init=0.25, staging=staging)
         check(res)
+
+
+def test_small_launches_skip_the_staging_and_give_the_same_bits():
+    """The library's own choice (no staging for a single wave of single-tile chunks) against
+    both forced modes: the arithmetic per coordinate is the same, so are the bits."""
+    w = di.Workload("small", "adam", 4, (4096, 1000, 37), "bf16", "normal1", lr=1e-2, K=(2, 3, 4), seed=5)
+    runs = [run_both(w, 8, staging=mode) for mode in (None, 0, 1)]
+    for r in runs:
+        check(r)
+    for r in runs[1:]:
+        for k in ("gx", "gu", "gv"):
+            assert np.array_equal(r[k], runs[0][k])
 
 
 @pytest.mark.parametrize("opt", ["adam", "adopt", "sgdm"])
