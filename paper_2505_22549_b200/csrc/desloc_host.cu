@@ -3,6 +3,7 @@
 // launcher that picks one kernel instantiation per step.  No torch types, no CPU compute path.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cmath>
 #include <cstdint>
 #include <cstdlib>
@@ -193,6 +194,7 @@ struct desloc_ctx {
     bool diag_valid = false;        // a diagnostics step has run since the workers last changed
     int64_t max_blocks = 0;         // test hook: cap on the grid (0 = one block per work item)
     int staging_mode = -1;          // test hook: -1 the library decides, 0 always stage, 1 never
+    std::vector<const void *> prepared;  // kernels whose shared-memory limit this context has raised
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t ev_entry = nullptr;
     cudaEvent_t ev_group[kHostGroups] = {};
@@ -340,10 +342,14 @@ int run_step(desloc_ctx *ctx, uint32_t mask, float lr_t, float clip_bound_t,
             const bool cap = lp.strides && ctx->max_blocks > 0 && lp.grid > ctx->max_blocks;
             return static_cast<unsigned>(cap ? ctx->max_blocks : lp.grid);
         };
-        e = desloc::prepare_launch(plan);
-        if (e != cudaSuccess) {
-            rc = cuda_fail(ctx, e);
-            break;
+        // (once per kernel: the attribute call costs a microsecond that a latency-bound step notices)
+        if (std::find(ctx->prepared.begin(), ctx->prepared.end(), plan.fn) == ctx->prepared.end()) {
+            e = desloc::prepare_launch(plan);
+            if (e != cudaSuccess) {
+                rc = cuda_fail(ctx, e);
+                break;
+            }
+            if (ctx->prepared.size() < ctx->prepared.capacity()) ctx->prepared.push_back(plan.fn);
         }
         if (!host_grads) {
             e = cudaLaunchKernel(plan.fn, dim3(capped(plan)),
@@ -491,6 +497,7 @@ int desloc_create(desloc_ctx **out, const desloc_config *cfg, float *const *x, f
     try {
         ctx->numel.assign(cfg->numel, cfg->numel + cfg->num_tensors);
         ctx->last_grads.assign(static_cast<size_t>(nptr), nullptr);
+        ctx->prepared.reserve(64);   // steps never allocate: beyond this the attribute is simply set again
         rchunks.resize(static_cast<size_t>(nrchunks));
         desloc::fill_chunks(cfg->numel, cfg->num_tensors, desloc::REDUCE_CHUNK_ELEMS, rchunks.data());
     } catch (const std::bad_alloc &) {
