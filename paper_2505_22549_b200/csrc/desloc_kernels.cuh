@@ -567,7 +567,7 @@ desloc_step_kernel(const __grid_constant__ StepArgs a) {
     // No factor on the gradient and no coordinate clip -- the common case -- takes a copy of the
     // inner loop without them (three instructions of about forty per coordinate: with eight
     // workers at sustained clocks 0.4-0.7 % of the step).  The fallback paths keep the one form.
-    const bool plain = a.gscale == nullptr && a.rho > 3.0e38f;
+    const bool plain = a.gscale == nullptr && a.rho > 3.4028235e38f;   // rho = +inf: clip off
     // Work items: chunks of all MT replicas; with MT = 1, (worker, chunk) pairs -- the single
     // replica and the local steps of more than MAX_MT workers.  One item per block as launched;
     // a smaller grid strides over the rest.
