@@ -156,7 +156,7 @@ struct WarpDiag {
 
 // One position (VEC elements) of all M workers.  `active` is false for the lanes a DIAG warp
 // carries past the end of the chunk: they touch no memory and contribute zeros to the sums.
-template <int OPT, typename GT, bool POST, int MASK, int VEC, bool DIAG>
+template <int OPT, typename GT, bool POST, int MASK, int VEC, bool DIAG, bool PLAIN = false>
 __device__ __forceinline__ void generic_position(const StepArgs &a, char *const (*sp)[GEN_MAX_M],
                                                  const float *sscale, long long e, bool active,
                                                  const WarpDiag<DIAG> &wd) {
@@ -187,7 +187,7 @@ __device__ __forceinline__ void generic_position(const StepArgs &a, char *const 
                     float gg = 0.f, dd = 0.f, xx = 0.f;
                     if (active) {
                         gg = sum_sq<VEC>(G[b]);
-                        const float sc = sscale[m0 + b];
+                        const float sc = PLAIN ? 1.f : sscale[m0 + b];
                         FV<VEC> D;
 #pragma unroll
                         for (int c = 0; c < VEC; ++c) {
@@ -196,7 +196,7 @@ __device__ __forceinline__ void generic_position(const StepArgs &a, char *const 
                             const float vp = SV ? vb.a[c] : vown;
                             const float xp = SX ? xb.a[c] : X[b].a[c];
                             float un, vn;
-                            state_update<OPT>(a, G[b].a[c] * sc, up, vp, vown, un, vn);
+                            state_update<OPT, PLAIN>(a, PLAIN ? G[b].a[c] : G[b].a[c] * sc, up, vp, vown, un, vn);
                             D.a[c] = direction<OPT>(a, un, vn);
                             X[b].a[c] = apply_step(a, xp, D.a[c]);
                             U[b].a[c] = un;
@@ -238,13 +238,13 @@ __device__ __forceinline__ void generic_position(const StepArgs &a, char *const 
                     float gg = 0.f, dd = 0.f, xx = 0.f;
                     if (active) {
                         gg = sum_sq<VEC>(G[b]);
-                        const float sc = sscale[m0 + b];
+                        const float sc = PLAIN ? 1.f : sscale[m0 + b];
                         FV<VEC> D;
 #pragma unroll
                         for (int c = 0; c < VEC; ++c) {
                             const float vown = OPT != OPT_SGDM ? V[b].a[c] : 0.f;
                             float un, vn;
-                            state_update<OPT>(a, G[b].a[c] * sc, U[b].a[c], vown, vown, un, vn);
+                            state_update<OPT, PLAIN>(a, PLAIN ? G[b].a[c] : G[b].a[c] * sc, U[b].a[c], vown, vown, un, vn);
                             U[b].a[c] = un;
                             V[b].a[c] = vn;
                             if constexpr (!P::D_NEEDS_MEAN) {
@@ -373,9 +373,17 @@ desloc_step_generic_kernel(const __grid_constant__ StepArgs a) {
         // DIAG warps run whole: lanes past the end take part in the shuffles with zeros
         if (!scalar_path) {
             const int n4 = ch.count >> 2;
-            for (int p = tid; DIAG ? (p - lane < n4) : (p < n4); p += BLOCK_THREADS)
-                generic_position<OPT, GT, POST, MASK, 4, DIAG>(a, sp, sscale, static_cast<long long>(p) * 4,
-                                                              p < n4, wd);
+            // (no gradient factor and no coordinate clip, the common case: a copy of the loop
+            // without them -- this kernel is bound by instruction issue)
+            if (a.gscale == nullptr && a.rho > 3.4028235e38f) {
+                for (int p = tid; DIAG ? (p - lane < n4) : (p < n4); p += BLOCK_THREADS)
+                    generic_position<OPT, GT, POST, MASK, 4, DIAG, true>(a, sp, sscale, static_cast<long long>(p) * 4,
+                                                                        p < n4, wd);
+            } else {
+                for (int p = tid; DIAG ? (p - lane < n4) : (p < n4); p += BLOCK_THREADS)
+                    generic_position<OPT, GT, POST, MASK, 4, DIAG>(a, sp, sscale, static_cast<long long>(p) * 4,
+                                                                  p < n4, wd);
+            }
             const int rem = ch.count & 3;
             if (DIAG ? (tid < 32 && rem > 0) : (tid < rem))
                 generic_position<OPT, GT, POST, MASK, 1, DIAG>(a, sp, sscale, (n4 << 2) + tid, tid < rem, wd);
