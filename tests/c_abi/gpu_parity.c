@@ -44,6 +44,39 @@ static float uniform_pm1(void) {   /* 64-bit LCG, top 24 bits -> [-1, 1) */
 #define DESLOC_OK_(call) do { int rc_ = (call); if (rc_ != DESLOC_OK) { \
     printf("%s -> %s (line %d)\n", #call, desloc_strerror(rc_), __LINE__); return 3; } } while (0)
 
+/* Steps per second a C caller gets on the latency-bound workload (N = 4096, two workers, fp32
+ * gradients, periods 4/8/16): 2000 back-to-back desloc_step() calls between two events.
+ * Printed for information, not checked. */
+static int eager_latency(void) {
+    const int64_t one[1] = {4096};
+    float *d;
+    CUDA_OK(cudaMalloc((void **)&d, 4 * 2 * 4096 * sizeof(float)));
+    CUDA_OK(cudaMemset(d, 0, 4 * 2 * 4096 * sizeof(float)));
+    float *x[2] = {d, d + 4096}, *u[2] = {d + 2 * 4096, d + 3 * 4096}, *v[2] = {d + 4 * 4096, d + 5 * 4096};
+    const void *g[2] = {d + 6 * 4096, d + 7 * 4096};
+    desloc_config cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.M = 2; cfg.num_tensors = 1; cfg.numel = one; cfg.opt = DESLOC_ADAM; cfg.grad_dtype = DESLOC_F32;
+    cfg.beta1 = 0.9f; cfg.beta2 = 0.999f; cfg.eps = 1e-8f; cfg.Kx = 4; cfg.Ku = 8; cfg.Kv = 16;
+    desloc_ctx *ctx = NULL;
+    DESLOC_OK_(desloc_create(&ctx, &cfg, x, u, v, 0));
+    cudaEvent_t e0, e1;
+    CUDA_OK(cudaEventCreate(&e0));
+    CUDA_OK(cudaEventCreate(&e1));
+    for (int64_t t = 0; t < 64; ++t) DESLOC_OK_(desloc_step(ctx, t, 1e-3f, 0.f, g, NULL, NULL));
+    CUDA_OK(cudaEventRecord(e0, NULL));
+    const int steps = 2000;
+    for (int64_t t = 64; t < 64 + steps; ++t) DESLOC_OK_(desloc_step(ctx, t, 1e-3f, 0.f, g, NULL, NULL));
+    CUDA_OK(cudaEventRecord(e1, NULL));
+    CUDA_OK(cudaEventSynchronize(e1));
+    float ms = 0.f;
+    CUDA_OK(cudaEventElapsedTime(&ms, e0, e1));
+    printf("eager desloc_step() from C, N = 4096, M = 2: %.2f us per step\n", 1e3 * ms / steps);
+    DESLOC_OK_(desloc_destroy(ctx));
+    cudaEventDestroy(e0); cudaEventDestroy(e1); cudaFree(d);
+    return 0;
+}
+
 int main(void) {
     int64_t off[NT], n = 0;
     for (int k = 0; k < NT; ++k) { off[k] = n; n += numel[k]; }
@@ -142,6 +175,8 @@ int main(void) {
     cudaFree(dx); cudaFree(du); cudaFree(dv); cudaFree(dg);
     free(hx); free(hu); free(hv); free(hg); free(gx); free(gu); free(gv);
     if (worst > 1e-5) { printf("gpu_parity: FAILED\n"); return 1; }
+    const int rc = eager_latency();
+    if (rc) return rc;
     printf("gpu_parity: ok\n");
     return 0;
 }
